@@ -1,0 +1,54 @@
+// Helpers of the C ABI and the dispatcher of step 5.
+#include "common.cuh"
+#include "stages.cuh"
+
+using namespace actqkv;
+
+extern "C" int actqkv_version(void) { return ACTQKV_VERSION; }
+
+extern "C" const char* actqkv_strerror(int status) {
+  switch (status) {
+    case ACTQKV_OK: return "ok";
+    case ACTQKV_ERR_NULL: return "a required pointer is NULL";
+    case ACTQKV_ERR_ALIGN: return "a data pointer is not 16-byte aligned";
+    case ACTQKV_ERR_SHAPE: return "unsupported shape or geometry";
+    case ACTQKV_ERR_DTYPE: return "unsupported dtype";
+    case ACTQKV_ERR_LAUNCH: return "the CUDA runtime refused the launch";
+    case ACTQKV_ERR_UNSUPPORTED: return "valid request this build cannot serve";
+    default: return "unknown actqkv status";
+  }
+}
+
+extern "C" int64_t actqkv_budget_state_bytes(const actqkv_config* cfg) {
+  return cfg ? int64_t(sizeof(double)) * (1 + 2 * int64_t(cfg->n_layers)) : 0;
+}
+
+extern "C" int32_t actqkv_n_candidates(const actqkv_config* cfg, int64_t p0) {
+  if (!cfg || cfg->block <= 0) return 0;
+  return make_geometry(p0, cfg->n_init, cfg->block, cfg->n_local_prev).n_cand;
+}
+
+extern "C" int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
+                                          const void* k_win, const void* v_win, int32_t n_tokens,
+                                          const void* k_pages, const void* v_pages, const int32_t* page_table,
+                                          const int64_t* pos0, const int32_t* sel_idx, const int32_t* sel_count,
+                                          void* out, float* lse, int32_t* status, void* stream) {
+  const Batch b = get_batch(batch);
+  int rc = check_config(cfg, b);
+  if (rc) return rc;
+  ACTQKV_REQUIRE_PTR(q);
+  ACTQKV_REQUIRE_PTR(k_win);
+  ACTQKV_REQUIRE_PTR(v_win);
+  ACTQKV_REQUIRE_PTR(k_pages);
+  ACTQKV_REQUIRE_PTR(v_pages);
+  ACTQKV_REQUIRE_PTR(out);
+  ACTQKV_OPTIONAL_PTR(lse);
+  if (!page_table || !pos0) return ACTQKV_ERR_NULL;
+  if (cfg->cap_blocks > 0 && (!sel_idx || !sel_count)) return ACTQKV_ERR_NULL;
+  if (n_tokens <= 0 || n_tokens > cfg->window) return ACTQKV_ERR_SHAPE;
+  AttnArgs a;
+  a.q = q; a.k_win = k_win; a.v_win = v_win; a.k_pages = k_pages; a.v_pages = v_pages;
+  a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
+  a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
+  return launch_attention_simt(cfg, b, a, reinterpret_cast<cudaStream_t>(stream));
+}

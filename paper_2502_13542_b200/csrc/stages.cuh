@@ -1,0 +1,44 @@
+// Internal launchers shared between translation units of the library.
+#pragma once
+#include "common.cuh"
+
+namespace actqkv {
+
+// Eq. 11 for one head, by one warp: theta = ln Z - sum_i e_i x_i / Z with
+// x_i = beta * s_i - max, e_i = exp(x_i), Z = sum_i e_i.  All lanes return theta.
+__device__ __forceinline__ float warp_entropy(const float* __restrict__ s, int n, float beta) {
+  if (n <= 0) return 0.f;
+  const int lane = threadIdx.x & 31;
+  float m = -INFINITY;
+  for (int i = lane; i < n; i += 32) m = fmaxf(m, beta * s[i]);
+  m = warp_max(m);
+  float z = 0.f, ex = 0.f;
+  for (int i = lane; i < n; i += 32) {
+    const float x = beta * s[i] - m;
+    const float e = expf(x);
+    z += e;
+    ex = fmaf(e, x, ex);
+  }
+  z = warp_sum(z);
+  ex = warp_sum(ex);
+  return fmaxf(logf(z) - ex / z, 0.f);
+}
+
+int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,
+                  const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
+                  cudaStream_t st);
+
+// Retrieval attention kernels: the general fp32-accumulate kernel and the tcgen05 kernel.
+struct AttnArgs {
+  const void *q, *k_win, *v_win, *k_pages, *v_pages;
+  const int32_t* page_table;
+  const int64_t* pos0;
+  const int32_t *sel_idx, *sel_count;
+  void* out;
+  float* lse;
+  int32_t* status;
+  int n_tokens;
+};
+int launch_attention_simt(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
+
+}  // namespace actqkv

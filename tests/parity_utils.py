@@ -1,0 +1,127 @@
+"""Shared machinery of the GPU parity tests: runs the oracle window by window on
+the seeded workload, keeps its state (incremental representative table), and
+compares the CUDA path's outputs with the tolerances the project states:
+
+  * selected block sets: identical, except blocks whose oracle score lies within
+    1e-3 (relative) of the cut-off score -- those are counted separately;
+  * activation bias, probe-query, scores (fp32): |a - b| <= 1e-4 * max(|b|, floor),
+    floor = 1 for cosines, 1e-3 * max|b| for phi / probe (phi -> 0 where q = mean);
+  * attention (bf16 in, fp32 accumulate): max abs err <= 2e-2, mean abs err <= 2e-3.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import actqkv_oracle as orc
+from paper_2502_13542_b200 import workloads as wl
+
+REL_TOL = 1e-4
+ATT_MAX_ABS = 2e-2
+ATT_MEAN_ABS = 2e-3
+NEAR_TIE_REL = 1e-3
+
+
+def rel_err_floor(got, want, floor):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    return float(np.max(np.abs(got - want) / np.maximum(np.abs(want), floor))) if want.size else 0.0
+
+
+def assert_rel(got, want, floor, what, tol=REL_TOL):
+    e = rel_err_floor(got, want, floor)
+    assert e <= tol, f"{what}: rel err {e:.3e} > {tol:.1e}"
+    return e
+
+
+def assert_phi_like(got, want, what):
+    want = np.asarray(want, np.float64)
+    floor = 1e-3 * max(float(np.max(np.abs(want))), 1e-30)
+    return assert_rel(got, want, floor, what)
+
+
+def attention_errors(got, want):
+    d = np.abs(np.asarray(got, np.float64) - np.asarray(want, np.float64))
+    return float(d.max()), float(d.mean())
+
+
+def assert_attention(got, want, what, dtype="bf16"):
+    """`got` is what the kernel stored (bf16 or fp32).  Compared against the raw fp64 oracle;
+    when the output is stored in bf16 the rounding of the stored value itself (|o| * 2^-9) is
+    part of the stated budget."""
+    mx, mean = attention_errors(got, want)
+    assert mx <= ATT_MAX_ABS and mean <= ATT_MEAN_ABS, f"{what}: max abs {mx:.3e}, mean abs {mean:.3e}"
+    return mx, mean
+
+
+def compare_selection(got_idx, got_count, oracle_res, what):
+    """got_idx [Hkv, cap] int32 (-1 padded), got_count int.  Returns number of near-tie
+    differences; asserts everything else is identical."""
+    near_diffs = 0
+    c = oracle_res["c"]
+    if got_count != c:
+        assert oracle_res["fragile"], f"{what}: count {got_count} != oracle {c} (B={oracle_res['b_real']})"
+        return -1
+    for g, want in enumerate(oracle_res["sel"]):
+        got = got_idx[g][:got_count]
+        assert np.all(got_idx[g][got_count:] == -1), f"{what}: head {g} tail not -1"
+        assert np.all(np.diff(got) > 0), f"{what}: head {g} not strictly ascending"
+        if np.array_equal(got, want):
+            continue
+        diff = set(got.tolist()) ^ set(want.tolist())
+        near = set(oracle_res["near"][g].tolist())
+        assert diff <= near, (f"{what}: head {g} differs outside the near-tie band: "
+                              f"{sorted(diff - near)} tau={oracle_res['tau'][g]}")
+        near_diffs += len(diff)
+    return near_diffs
+
+
+class OracleRunner:
+    """The oracle's view of one (sequence, layer): state + incremental representative table."""
+
+    def __init__(self, spec: wl.WorkloadSpec, layer: int = 0, chain: orc.BudgetChain | None = None,
+                 beta: float = 1.0, thetabar_mode: str = "streaming", repr_mode="chunk_mean", agg="mean"):
+        self.spec, self.layer, self.beta = spec, layer, beta
+        self.repr_mode, self.agg = repr_mode, agg
+        self.state = orc.LayerState(spec.n_q_heads, spec.n_kv_heads, spec.head_dim)
+        self.chain = chain or orc.BudgetChain(spec.n_layers, spec.k_blocks, spec.cap_blocks, thetabar_mode)
+        self.table = np.zeros((spec.n_kv_heads, 0, spec.n_repr, spec.head_dim))
+
+    def _extend_table(self, n_blocks):
+        sp = self.spec
+        have = self.table.shape[1]
+        if n_blocks <= have:
+            return
+        new = np.zeros((sp.n_kv_heads, n_blocks - have, sp.n_repr, sp.head_dim))
+        for g in range(sp.n_kv_heads):
+            for b in range(have, n_blocks):
+                lo = sp.n_init + b * sp.block
+                new[g, b - have] = orc.build_representatives(self.state.k_cache[lo:lo + sp.block, g, :],
+                                                             sp.n_repr, sp.dtype, self.repr_mode)
+        self.table = np.concatenate([self.table, new], axis=1)
+
+    def complete_blocks(self):
+        sp = self.spec
+        n_tok = self.state.k_cache.shape[0]
+        return max(0, (n_tok - sp.n_init) // sp.block)
+
+    def step(self, q, k, v, attention=True, theta_all=None, layer_in_model=None):
+        sp = self.spec
+        self._extend_table(self.complete_blocks())
+        res = orc.window_retrieval(self.state, self.chain, self.layer if layer_in_model is None else layer_in_model,
+                                   q, k, v, n_init=sp.n_init, block=sp.block,
+                                   n_repr=sp.n_repr, dtype=sp.dtype, n_local_prev=sp.n_local_prev,
+                                   beta=self.beta, repr_mode=self.repr_mode, agg=self.agg,
+                                   attention=attention, theta_all=theta_all, repr_table=self.table)
+        self._extend_table(self.complete_blocks())
+        return res
+
+
+def to_device(x, spec, device="cuda"):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(device)
+    return t.to(torch.bfloat16) if spec.dtype == "bf16" else t
+
+
+def to_numpy(t):
+    import torch
+    return t.detach().to(torch.float32).cpu().numpy() if t.dtype != torch.float64 else t.detach().cpu().numpy()

@@ -1,0 +1,262 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs."""
+import numpy as np
+import pytest
+
+from oracle import actqkv_oracle as orc
+from paper_2502_13542_b200 import workloads as wl
+from tests import parity_utils as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2502_13542_b200 import binding
+    return binding
+
+
+def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.0, stop_after=None):
+    """Runs every window of a single-layer workload through RetrievalState.step() and the
+    oracle; compares every intermediate.  Returns summary statistics."""
+    import torch
+    cfg = B.make_config(spec, beta=beta)
+    n_pages = cfg.n_phys_pages
+    pt = wl.shuffled_page_table(spec, spec.context)
+    st = B.RetrievalState(cfg, page_table=pt[None, :], keep_phi=True)
+    o_run = pu.OracleRunner(spec, beta=beta)
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=cfg.torch_dtype, device="cuda")
+    lse = torch.zeros(spec.n_q_heads, spec.window, dtype=torch.float32, device="cuda")
+    stats = dict(near=0, worst_att=0.0, worst_att_mean=0.0, worst_rel=0.0, fragile=0)
+    last = spec.n_windows if stop_after is None else stop_after
+    for t in range(last):
+        q = wl.gen_q(spec, 0, t)
+        k, v = wl.gen_kv(spec, 0, t)
+        p0 = t * spec.window
+        assert st.host_pos0[0] == p0
+        do_att = t in windows_with_attention
+        res = o_run.step(q, k, v, attention=do_att)
+        st.step(pu.to_device(q[None], spec), pu.to_device(k[None], spec), pu.to_device(v[None], spec),
+                out, lse=lse, fused=fused)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0, f"window {t}: device status {int(st.status.item())}"
+        if not (check_every or do_att):
+            continue
+        tag = f"{spec.name} window {t}"
+        n = res["n"]
+        assert int(st.n_cand.item()) == n
+        # step 1: statistics and activation bias
+        pu.assert_rel(pu.to_numpy(st.stats_mean[0]), res["zbar"], 1e-3 * np.abs(res["zbar"]).max() + 1e-30, tag + " mean")
+        cnt = int(st.stats_count[0, 0].item())
+        assert cnt == (t + 1) * spec.window
+        var_gpu = pu.to_numpy(st.stats_m2[0]) / max(cnt - 1, 1)
+        pu.assert_rel(var_gpu, res["sigma2"], 1e-30, tag + " variance")
+        e1 = pu.assert_phi_like(pu.to_numpy(st.phi_l1[0]).T, res["phi_l1"], tag + " phi_l1")
+        e2 = pu.assert_phi_like(pu.to_numpy(st.phi_full[0]), res["phi"], tag + " phi")
+        # step 2: probes
+        e3 = pu.assert_phi_like(pu.to_numpy(st.probe_qh[0]), res["probe_qh"], tag + " probe_qh")
+        e4 = pu.assert_phi_like(pu.to_numpy(st.probe_kv[0]), res["probe_kv"], tag + " probe_kv")
+        # step 3: scores and density
+        e5 = 0.0
+        if n:
+            e5 = pu.assert_rel(pu.to_numpy(st.scores[0, :, :n]), res["scores"], 1.0, tag + " scores")
+            pu.assert_rel(pu.to_numpy(st.theta[0]), res["theta"], 1e-30, tag + " theta")
+        stats["worst_rel"] = max(stats["worst_rel"], e1, e2, e3, e4, e5)
+        # step 4: selection
+        nd = pu.compare_selection(pu.to_numpy(st.sel_idx[0]).astype(np.int64), int(st.sel_count.item()), res, tag)
+        if nd < 0:
+            stats["fragile"] += 1
+        else:
+            stats["near"] += nd
+        # step 5: attention (only meaningful when the selected sets agree)
+        if do_att and nd == 0:
+            mx, mean = pu.assert_attention(pu.to_numpy(out), res["out"], tag + " attention", spec.dtype)
+            stats["worst_att"] = max(stats["worst_att"], mx)
+            stats["worst_att_mean"] = max(stats["worst_att_mean"], mean)
+            pu.assert_rel(pu.to_numpy(lse), res["lse"], 1.0, tag + " lse", tol=2e-3)
+        # step 6: table rows of the blocks completed so far are bit-identical, pages hold the cache
+        nb = o_run.complete_blocks()
+        tab = pu.to_numpy(st.repr_k[0, :, :nb]).astype(np.float64)
+        assert np.array_equal(tab, o_run.table[:, :nb]), tag + " representative table"
+        inv = 1.0 / np.sqrt((o_run.table[:, :nb] ** 2).sum(axis=-1))
+        pu.assert_rel(pu.to_numpy(st.repr_inv_norm[0, :, :nb]), inv, 1e-30, tag + " inv norms", tol=1e-5)
+    # the pages hold exactly the appended cache
+    n_tok = last * spec.window
+    kp = pu.to_numpy(st.k_pages[0])
+    vp = pu.to_numpy(st.v_pages[0])
+    want_k = wl.to_pages(spec, o_run.state.k_cache[:n_tok], pt, n_pages)
+    want_v = wl.to_pages(spec, o_run.state.v_cache[:n_tok], pt, n_pages)
+    used = pt[: n_tok // spec.page_tokens]
+    assert np.array_equal(kp[used], want_k[used]) and np.array_equal(vp[used], want_v[used])
+    return stats, o_run, st
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_tiny_config_every_window(B, fused):
+    spec = wl.tiny_pr1()
+    stats, o_run, st = _run_sweep(B, spec, set(range(spec.n_windows)), fused)
+    print("tiny sweep", stats)
+    assert stats["fragile"] == 0
+    # planted blocks retrieved by the CUDA path at the target window, as by the oracle
+    sel = pu.to_numpy(st.sel_idx[0]).astype(int)
+    for g in range(spec.n_kv_heads):
+        assert set(wl.planted_blocks(spec, 0)[g]) <= set(sel[g])
+
+
+def test_tiny_all_blocks_equals_full_causal_attention(B):
+    """Budget covering every block: the CUDA attention must equal brute-force causal attention."""
+    import torch
+    spec = wl.tiny_pr1().replace(k_blocks=64, cap_blocks=64)
+    cfg = B.make_config(spec)
+    st = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :])
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    ks, vs = [], []
+    for t in range(6):
+        q = wl.gen_q(spec, 0, t)
+        k, v = wl.gen_kv(spec, 0, t)
+        ks.append(k); vs.append(v)
+        st.step(pu.to_device(q[None], spec), pu.to_device(k[None], spec), pu.to_device(v[None], spec), out)
+        torch.cuda.synchronize()
+        if t in (0, 1, 5):
+            want = orc.full_causal_attention(q[-40:], np.concatenate(ks), np.concatenate(vs), t * spec.window + spec.window - 40)
+            got = pu.to_numpy(out)[-40:]
+            assert np.abs(got - want).max() < 1e-4
+    assert int(st.status.item()) == 0
+
+
+def test_llama_layer_32k_sampled_windows(B):
+    """LLaMA3-8B-shaped layer, bf16 paged cache, 32k context: steps 1-4 and 6 at every window,
+    attention against the oracle at windows {0, 1, 2, 31, 63}."""
+    spec = wl.llama3_8b_layer()
+    stats, o_run, st = _run_sweep(B, spec, {0, 1, 2, 31, 63}, fused=True)
+    print("llama 32k sweep", stats)
+    sel = pu.to_numpy(st.sel_idx[0]).astype(int)
+    for g in range(spec.n_kv_heads):
+        assert set(wl.planted_blocks(spec, 0)[g]) <= set(sel[g])
+
+
+def test_select_cutoff_bit_exact_on_oracle_scores(B):
+    """The selection kernel alone, fed fp32 scores from the host: identical to a stable sort,
+    including exact ties, NaN, n < c and n = 0."""
+    import torch
+    spec = wl.llama3_8b_layer().replace(cap_blocks=64, k_blocks=48)
+    rng = np.random.default_rng(7)
+    for n in (0, 1, 5, 48, 49, 251, 1019, 2000):
+        cfg = B.make_config(spec, n_cap=2048)
+        s = rng.standard_normal((8, 2048)).astype(np.float32)
+        s[:, 10:40] = np.float32(0.25)                                   # a run of exact ties
+        s[3, 7] = np.nan
+        s[4, :] = np.round(s[4, :] * 4) / 4                              # heavy ties everywhere
+        scores = torch.from_numpy(s).cuda()[None]
+        theta = torch.full((1, 8), 5.0, device="cuda")
+        n_cand = torch.tensor([n], dtype=torch.int32, device="cuda")
+        state = torch.zeros(1, B.budget_state_bytes(cfg) // 8, dtype=torch.float64, device="cuda")
+        sel_idx = torch.zeros(1, 8, 64, dtype=torch.int32, device="cuda")
+        sel_count = torch.zeros(1, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.select_cutoff(cfg, None, scores, theta, n_cand, state, sel_idx, sel_count, None, status)
+        torch.cuda.synchronize()
+        c = int(sel_count.item())
+        assert c == min(48, n) and int(status.item()) == 0
+        got = sel_idx[0].cpu().numpy()
+        for g in range(8):
+            want, _, _ = orc.select_blocks(s[g, :n], c)
+            assert np.array_equal(got[g, :c], want), (n, g)
+            assert np.all(got[g, c:] == -1)
+
+
+def test_budget_chain_32_layers_matches_oracle(B):
+    """Eq. 12 over a 32-layer batch, several steps, both theta-bar readings, with a sharpened
+    softmax (beta = 32) so that the per-layer counts really differ and hit the cap."""
+    import torch
+    spec = wl.tiny_stack32()
+    L, Hkv, n = 32, spec.n_kv_heads, 29
+    for mode_name, mode in (("streaming", 0), ("alg1", 1)):
+        cfg = B.make_config(spec, beta=32.0, thetabar_mode=mode, n_cap=32)
+        chain = orc.BudgetChain(L, spec.k_blocks, spec.cap_blocks, mode_name)
+        state = torch.zeros(1, B.budget_state_bytes(cfg) // 8, dtype=torch.float64, device="cuda")
+        batch = B.Batch(1, L, 0)
+        rng = np.random.default_rng(11)
+        for step in range(4):
+            s = (rng.standard_normal((L, Hkv, 32)) * rng.uniform(0.02, 0.5, (L, 1, 1))).astype(np.float32)
+            s = np.clip(s, -1, 1)
+            scores = torch.from_numpy(s).cuda()
+            theta = torch.zeros(L, Hkv, device="cuda")
+            n_cand = torch.tensor([n], dtype=torch.int32, device="cuda")
+            sel_idx = torch.zeros(L, Hkv, spec.cap_blocks, dtype=torch.int32, device="cuda")
+            sel_count = torch.zeros(L, dtype=torch.int32, device="cuda")
+            real = torch.zeros(L, device="cuda")
+            probe = torch.zeros(L, Hkv, spec.head_dim, device="cuda")
+            # density from the kernel (score_blocks' second half is exercised through select's fused path)
+            th_or = np.stack([orc.information_density(s[l, :, :n], 32.0) for l in range(L)])
+            theta.copy_(torch.from_numpy(th_or.astype(np.float32)))
+            B.select_cutoff(cfg, batch, scores, theta, n_cand, state, sel_idx, sel_count, real, None)
+            torch.cuda.synchronize()
+            got_c = sel_count.cpu().numpy()
+            th_layer = th_or.astype(np.float32).astype(np.float64).mean(axis=1)
+            want_c, frag = [], []
+            for l in range(L):
+                c, b_real, fragile = chain.grant(l, th_or[l], n, th_layer)
+                want_c.append(c); frag.append(fragile)
+                assert abs(float(real[l]) - b_real) <= 1e-4 * max(1.0, abs(b_real))
+            assert not any(frag)
+            assert got_c.tolist() == want_c, (mode_name, step)
+            assert len(set(want_c)) > 2                                   # counts really vary
+            for l in range(L):
+                for g in range(Hkv):
+                    want, _, _ = orc.select_blocks(s[l, g, :n], want_c[l])
+                    assert np.array_equal(sel_idx[l, g, :want_c[l]].cpu().numpy(), want)
+        assert abs(float(state[0, 0]) - chain.b_rem) < 1e-9
+
+
+def test_edge_cases_and_errors(B):
+    import torch
+    spec = wl.tiny_pr1()
+    cfg = B.make_config(spec)
+    st = B.RetrievalState(cfg)
+    q = torch.zeros(1, 256, 4, 64, device="cuda")
+    with pytest.raises(B.ActQKVError):                                  # misaligned pointer
+        B.activation_bias(cfg, None, q.view(-1)[1:].contiguous()[: 256 * 4 * 64 - 4].view(-1), 256, st.stats_count,
+                          st.stats_mean, st.stats_m2, st.phi_l1)
+    with pytest.raises(B.ActQKVError):                                  # n_tokens > window
+        B.activation_bias(cfg, None, q, 512, st.stats_count, st.stats_mean, st.stats_m2, st.phi_l1)
+    bad = B.make_config(spec)
+    bad.head_dim = 96
+    with pytest.raises(B.ActQKVError):
+        B.activation_bias(bad, None, q, 256, st.stats_count, st.stats_mean, st.stats_m2, st.phi_l1)
+    # out-of-range page index: flagged, not dereferenced
+    st2 = B.RetrievalState(cfg, page_table=np.full((1, cfg.max_pages), 10 ** 6, np.int32))
+    out = torch.zeros(256, 4, 64, device="cuda")
+    k = torch.randn(1, 256, 2, 64, device="cuda")
+    st2.step(torch.randn(1, 256, 4, 64, device="cuda"), k, k, out)
+    torch.cuda.synchronize()
+    assert int(st2.status.item()) & B.DEV_BAD_PAGE
+    # constant queries: zero variance -> floor, uniform weights, probe = the query itself
+    st3 = B.RetrievalState(cfg)
+    qc = torch.full((1, 256, 4, 64), 0.5, device="cuda")
+    B.bias_probe(cfg, None, qc, 256, st3.stats_count, st3.stats_mean, st3.stats_m2, st3.phi_l1, None,
+                 st3.probe_qh, st3.probe_kv, st3.status)
+    torch.cuda.synchronize()
+    assert torch.all(st3.phi_l1 == 0) and torch.allclose(st3.probe_kv, torch.full_like(st3.probe_kv, 0.5))
+    # a ragged step (n_tokens not a multiple of anything) and a single decode token
+    spec_r = spec
+    o_run = pu.OracleRunner(spec_r)
+    st4 = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec_r, spec_r.context)[None, :])
+    for t in range(3):
+        qn = wl.gen_q(spec_r, 0, t); kn, vn = wl.gen_kv(spec_r, 0, t)
+        o_run.step(qn, kn, vn, attention=False)
+        st4.step(pu.to_device(qn[None], spec_r), pu.to_device(kn[None], spec_r), pu.to_device(vn[None], spec_r), out)
+    for nt in (37, 1):
+        qn = wl.gen_q(spec_r, 0, 3)[:nt]; kn, vn = wl.gen_kv(spec_r, 0, 3)
+        kn, vn = kn[:nt], vn[:nt]
+        res = o_run.step(qn, kn, vn, attention=True)
+        o = torch.zeros(nt, 4, 64, device="cuda")
+        st4.step(pu.to_device(qn[None], spec_r), pu.to_device(kn[None], spec_r), pu.to_device(vn[None], spec_r), o,
+                 n_tokens=nt)
+        torch.cuda.synchronize()
+        assert pu.compare_selection(pu.to_numpy(st4.sel_idx[0]).astype(np.int64), int(st4.sel_count.item()), res,
+                                    f"ragged {nt}") == 0
+        pu.assert_attention(pu.to_numpy(o), res["out"], f"ragged step of {nt} tokens")
+    assert int(st4.status.item()) == 0
