@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the ActQKV per-window retrieval path on B200.
+
+One "step" = the whole hot path (bias+probe -> score -> cut-off/select -> attention -> append)
+for one window of W queries of one layer at the last window of a 32k-token prefill of the
+LLaMA3-8B-shaped workload.  Metric: prefill retrieval tokens/s/layer = W / step time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Cold L2: consecutive steps run on different, physically distinct copies of the layer state
+(caches, tables, inputs; > 2x L2 in total), so nothing a step reads is left in L2 by the
+previous one.  Under torchrun every rank runs its own copies (independent layers: weak
+scaling, no collective on the data path); rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "prefill retrieval tokens/sec/layer at 32k ctx"
+UNIT = "tokens/s/layer"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period=0.05):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(
+                nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                     0x4: "sw_power_cap", 0x80: "hw_power_brake"}
+            for bit, name in names.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self._stop_evt.is_set():
+            self.sample()
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def attention_flops(spec, p0, c_blocks):
+    """Causal-counted useful flops of one window's attention (4*D per query-key pair)."""
+    from paper_2502_13542_b200 import workloads as wl
+    n = wl.n_candidates(spec, p0)
+    n_past = (spec.n_init + c_blocks * spec.block + (p0 - (spec.n_init + n * spec.block))) if p0 > spec.n_init else p0
+    W = spec.window
+    pairs = W * n_past + W * (W + 1) // 2
+    return 4.0 * spec.head_dim * spec.n_q_heads * pairs
+
+
+def stage_bytes(spec, p0):
+    """Algorithmic HBM bytes of the memory-bound stages of one window (dtype bf16 = 2 B)."""
+    from paper_2502_13542_b200 import workloads as wl
+    e = 2 if spec.dtype == "bf16" else 4
+    n = wl.n_candidates(spec, p0)
+    W, Hq, Hkv, D, r = spec.window, spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.n_repr
+    return {
+        "bias_probe": W * Hq * D * e + 3 * Hq * D * 4 + Hq * W * 4,
+        "score": n * Hkv * r * D * e + n * Hkv * r * 4 + n * Hkv * 4,
+        "select": n * Hkv * 4 + spec.cap_blocks * Hkv * 4,
+        "append": 2 * 2 * W * Hkv * D * e,
+    }
+
+
+# ------------------------------------------------------------------------------------------
+def build_states(spec, n_copies, device):
+    """Prefills one layer up to the last window on the GPU, then clones the state into
+    n_copies physically distinct copies.  Returns (cfg, states, inputs of the last window)."""
+    import torch
+    from paper_2502_13542_b200 import binding as B
+    from paper_2502_13542_b200 import workloads as wl
+    from tests import parity_utils as pu
+
+    cfg = B.make_config(spec, out_dtype=B.BF16)
+    base = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :], device=device)
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=device)
+    T = spec.n_windows
+    for t in range(T - 1):
+        q = pu.to_device(wl.gen_q(spec, 0, t)[None], spec, device)
+        k, v = wl.gen_kv(spec, 0, t)
+        base.step(q, pu.to_device(k[None], spec, device), pu.to_device(v[None], spec, device), out)
+    torch.cuda.synchronize()
+    q = pu.to_device(wl.gen_q(spec, 0, T - 1)[None], spec, device)
+    k, v = wl.gen_kv(spec, 0, T - 1)
+    k, v = pu.to_device(k[None], spec, device), pu.to_device(v[None], spec, device)
+    states, inputs = [], []
+    names = ["stats_count", "stats_mean", "stats_m2", "repr_k", "repr_inv_norm", "budget_state", "k_pages",
+             "v_pages", "probe_kv", "probe_qh"]
+    for i in range(n_copies):
+        st = B.RetrievalState(cfg, page_table=base.page_table.cpu().numpy(), device=device)
+        for nme in names:
+            getattr(st, nme).copy_(getattr(base, nme))
+        st.set_positions(base.host_pos0)
+        states.append(st)
+        inputs.append((q.clone(), k.clone(), v.clone(), torch.zeros_like(out)))
+    return cfg, states, inputs
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_13542_b200 import binding as B
+    from paper_2502_13542_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    spec = wl.llama3_8b_layer()
+    p0 = (spec.n_windows - 1) * spec.window
+    n_copies = args.copies
+    cfg, states, inputs = build_states(spec, n_copies, device)
+    peaks = load_peaks()
+
+    def one_step(i, events=None):
+        st = states[i % n_copies]
+        q, k, v, out = inputs[i % n_copies]
+        b = st.batch
+        calls = (
+            ("bias_probe", lambda: B.bias_probe(cfg, b, q, spec.window, st.stats_count, st.stats_mean, st.stats_m2,
+                                                st.phi_l1, None, st.probe_qh, st.probe_kv, st.status)),
+            ("score_select", lambda: B.score_select(cfg, b, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand,
+                                                    st.budget_state, st.scores, st.theta, st.sel_idx, st.sel_count,
+                                                    st.budget_real, st.status)),
+            ("attention", lambda: B.retrieval_attention(cfg, b, q, k, v, spec.window, st.k_pages, st.v_pages,
+                                                        st.page_table, st.pos0, st.sel_idx, st.sel_count, out, None,
+                                                        st.status)),
+            ("append", lambda: B.append_window(cfg, b, k, v, spec.window, st.pos0, st.k_pages, st.v_pages,
+                                               st.page_table, st.repr_k, st.repr_inv_norm, st.status)),
+        )
+        for name, fn in calls:
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                events.setdefault(name, []).append((e0, e1))
+            else:
+                fn()
+
+    launches_per_step = 6   # bias_probe, score, cut-off chain, select, attention, append
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        one_step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        one_step(args.warmup + i)
+    e1.record()
+    sampler.sample()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * spec.window / (ms_step * 1e-3)
+
+    # instrumented pass: per-stage device time with events around each call
+    events = {}
+    for i in range(args.steps):
+        one_step(args.warmup + i, events)
+    torch.cuda.synchronize()
+    stage_us = {k: 1e3 * float(np.mean([a.elapsed_time(b) for a, b in v])) for k, v in events.items()}
+    assert all(int(st.status.item()) == 0 for st in states), "device status set during the bench"
+
+    c_sel = int(states[0].sel_count.item())
+    flops = attention_flops(spec, p0, c_sel)
+    att_tflops = flops / (stage_us["attention"] * 1e-6) / 1e12
+    peak = peaks["bf16_tflops"]
+    roofline = {"bound": "tensor", "kernel": "retrieval_attention", "achieved": att_tflops, "peak": peak,
+                "unit": "TFLOP/s", "frac": att_tflops / peak, "traffic": None,
+                "peak_source": peaks["source"] + " burst bf16 (cuBLAS)", "flops_per_launch": flops}
+    sb = stage_bytes(spec, p0)
+    stages = {k: {"us": v} for k, v in stage_us.items()}
+    stages["bias_probe"]["GBps"] = sb["bias_probe"] / stage_us["bias_probe"] / 1e3
+    stages["score_select"]["GBps"] = (sb["score"] + sb["select"]) / stage_us["score_select"] / 1e3
+    stages["append"]["GBps"] = sb["append"] / stage_us["append"] / 1e3
+    stages["attention"]["TFLOPs"] = att_tflops
+
+    # end to end through the public API with host buffers (pinned), copies inside the timed region
+    q, k, v, out = inputs[0]
+    hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
+    ho = torch.empty_like(out, device="cpu").pin_memory()
+    e2e_steps = max(3, min(args.steps, 200))
+
+    def e2e_step(i):
+        st = states[i % n_copies]
+        dq, dk, dv, dout = inputs[i % n_copies]
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+        one_step(i)
+        ho.copy_(dout, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(3 + i)
+    t_e2e = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([t_e2e], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e = float(t.item())
+    e2e = {"value": world * spec.window * e2e_steps / t_e2e, "unit": UNIT,
+           "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
+           "d2h_bytes_per_step": int(ho.numel()) * 2, "steps": e2e_steps}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "llama3_8b_layer_32k: last window (p0=32256) of a 32768-token prefill, "
+                               "Hq=32 Hkv=8 D=128 W=512 B=128 r=4 n_init=128 k=cap=32, bf16 16-token pages",
+                   "cold_l2": f"{n_copies} distinct layer-state copies rotated (inputs larger than L2)",
+                   "selected_blocks": c_sel, "parallelism": f"independent layers x{world}"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline, "stages": stages,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(spec, budget_s=args.cpu_budget)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------
+def _oracle_sample(spec, st_cache, q, k, v, heads):
+    """Times the oracle on one window: steps 1-4 in full, attention for `heads` KV heads."""
+    from oracle import actqkv_oracle as orc
+    state, chain, table = st_cache
+    t0 = time.perf_counter()
+    s2 = state.stats.copy()
+    s2.update(q)
+    phi, a = orc.activation_bias(q, s2.mean, s2.variance())
+    pq = orc.probe_query(q, a)
+    pkv = orc.kv_head_probe(pq, spec.n_kv_heads)
+    p0 = state.k_cache.shape[0]
+    n = orc.n_candidate_blocks(p0, spec.n_init, spec.block, spec.n_local_prev)
+    s = orc.block_scores(pkv, table[:, :n])
+    theta = orc.information_density(s)
+    c = min(spec.k_blocks, n)
+    sel = [orc.select_blocks(s[g], c)[0] for g in range(spec.n_kv_heads)]
+    t1 = time.perf_counter()
+    G = spec.group
+    for g in heads:
+        orc.retrieval_attention(q[:, g * G:(g + 1) * G], k[:, g:g + 1], v[:, g:g + 1], state.k_cache[:, g:g + 1],
+                                state.v_cache[:, g:g + 1], p0, [sel[g]], spec.n_init, spec.block, spec.n_local_prev)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def _oracle_state(spec):
+    from oracle import actqkv_oracle as orc
+    from paper_2502_13542_b200 import workloads as wl
+    from tests import parity_utils as pu
+    run = pu.OracleRunner(spec)
+    T = spec.n_windows
+    for t in range(T - 1):
+        run.state.stats.update(wl.gen_q(spec, 0, t))
+        k, v = wl.gen_kv(spec, 0, t)
+        run.state.k_cache, run.state.v_cache = orc.append_window(run.state.k_cache, run.state.v_cache, k, v)
+    run._extend_table(run.complete_blocks())
+    q = wl.gen_q(spec, 0, T - 1)
+    k, v = wl.gen_kv(spec, 0, T - 1)
+    return (run.state, run.chain, run.table), q, k, v
+
+
+def cpu_baseline(spec, budget_s=20.0):
+    import torch
+    st, q, k, v = _oracle_state(spec)
+    t14, tatt = _oracle_sample(spec, st, q, k, v, heads=[0])
+    est = t14 + tatt * spec.n_kv_heads
+    cores = int(os.environ.get("OMP_NUM_THREADS", 0)) or torch.get_num_threads()
+    return {"value": spec.window / est, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"steps 1-4 in full ({t14:.2f} s) + attention of 1 of {spec.n_kv_heads} KV heads "
+                      f"({tatt:.2f} s), attention time scaled by {spec.n_kv_heads}"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2502_13542_b200 import workloads as wl
+    spec = wl.llama3_8b_layer()
+    st, q, k, v = _oracle_state(spec)
+    times = []
+    for i in range(args.warmup + args.steps):
+        t14, tatt = _oracle_sample(spec, st, q, k, v, heads=[i % spec.n_kv_heads])
+        if i >= args.warmup:
+            times.append(t14 + tatt * spec.n_kv_heads)
+    ms = 1e3 * float(np.mean(times))
+    import torch
+    val = spec.window / (ms * 1e-3)
+    cores = torch.get_num_threads()
+    sample = "each step: oracle steps 1-4 in full + attention of 1 of 8 KV heads, attention time scaled by 8"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama3_8b_layer_32k: last window (p0=32256) of a 32768-token prefill (CPU oracle)"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--copies", type=int, default=8)
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        args.steps = min(args.steps, 5)
+        args.warmup = min(args.warmup, 1)
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -101,6 +101,7 @@ typedef struct actqkv_config {
   float beta;            /* softmax(beta * s) in Eq. 11; 1 = the paper                    */
   float sm_scale;        /* attention scale; 0 => 1/sqrt(D)                               */
   float var_eps;         /* floor on sigma^2 in Eq. 7; 0 => 1e-12                         */
+  int32_t out_dtype;     /* element type of the attention output: ACTQKV_F32 | ACTQKV_BF16 */
 } actqkv_config;
 
 typedef struct actqkv_batch {
@@ -125,7 +126,7 @@ int32_t actqkv_n_candidates(const actqkv_config* cfg, int64_t p0);
  * then phi[j,h,c] = (q[j,h,c] - mean[h,c])^2 / max(var[h,c], var_eps) and the token
  * indicator phi_l1[h,j] = sum_c phi[j,h,c].
  *   q          [U][n_tokens][Hq][D]  dtype, in
- *   stats_count[U]                   int64, in/out (tokens merged so far)
+ *   stats_count[U][Hq]               int64, in/out (tokens merged so far)
  *   stats_mean [U][Hq][D]            fp32, in/out
  *   stats_m2   [U][Hq][D]            fp32, in/out
  *   phi_l1     [U][Hq][n_tokens]     fp32, out
@@ -196,7 +197,7 @@ int actqkv_score_select(const actqkv_config* cfg, const actqkv_batch* batch, con
  *   page_table   [n_seq][max_pages]     int32 in (logical page -> physical page)
  *   pos0         [n_seq]                int64 in (device): p0 of each sequence
  *   sel_idx, sel_count                  as written by select_cutoff
- *   out          [U][n_tokens][Hq][D]   dtype out
+ *   out          [U][n_tokens][Hq][D]   cfg->out_dtype out
  *   lse          [U][Hq][n_tokens]      fp32 out, may be NULL (natural-log sum of exp)
  * bf16, D = 128, B = 128, n_tokens and p0 multiples of 128 run on the tcgen05 tensor-core
  * kernel; every other shape runs on the general fp32-accumulate kernel. */

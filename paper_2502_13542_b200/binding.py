@@ -37,11 +37,15 @@ class Config(C.Structure):
         "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "window", "block", "n_repr", "page_tokens",
         "n_init", "n_local_prev", "k_blocks", "cap_blocks", "dtype", "stats_mode", "repr_mode",
         "agg_mode", "thetabar_mode", "n_cap", "max_pages", "n_phys_pages")] + [
-        ("beta", C.c_float), ("sm_scale", C.c_float), ("var_eps", C.c_float)]
+        ("beta", C.c_float), ("sm_scale", C.c_float), ("var_eps", C.c_float), ("out_dtype", C.c_int32)]
 
     @property
     def torch_dtype(self):
         return torch.bfloat16 if self.dtype == BF16 else torch.float32
+
+    @property
+    def torch_out_dtype(self):
+        return torch.bfloat16 if self.out_dtype == BF16 else torch.float32
 
     @property
     def group(self):
@@ -176,7 +180,7 @@ def append_window(cfg, batch, k_win, v_win, n_tokens, pos0, k_pages, v_pages, pa
 # ----------------------------------------------------------------------------
 def make_config(spec, *, n_cap=None, max_pages=None, n_phys_pages=None, beta=1.0,
                 stats_mode=STATS_CUMULATIVE, repr_mode=REPR_CHUNK_MEAN, agg_mode=AGG_MEAN,
-                thetabar_mode=THETABAR_STREAMING, max_context=None) -> Config:
+                thetabar_mode=THETABAR_STREAMING, max_context=None, out_dtype=None) -> Config:
     """Config for a `workloads.WorkloadSpec`-like object (any object with the same fields)."""
     ctx = max_context if max_context is not None else spec.context + spec.decode_steps
     pages = -(-ctx // spec.page_tokens)
@@ -192,6 +196,7 @@ def make_config(spec, *, n_cap=None, max_pages=None, n_phys_pages=None, beta=1.0
     cfg.max_pages = max_pages if max_pages is not None else pages
     cfg.n_phys_pages = n_phys_pages if n_phys_pages is not None else pages
     cfg.beta, cfg.sm_scale, cfg.var_eps = beta, 0.0, 0.0
+    cfg.out_dtype = cfg.dtype if out_dtype is None else out_dtype
     return cfg
 
 

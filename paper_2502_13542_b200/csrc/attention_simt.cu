@@ -27,7 +27,7 @@ struct SimtParams {
   float scale_log2;
 };
 
-template <typename T, int D>
+template <typename T, typename TO, int D>
 __global__ void __launch_bounds__(kWarps * 32) attention_simt_kernel(SimtParams p) {
   __shared__ float Ks[kChunk][D + 1];
   __shared__ float Vs[kChunk][D];
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(kWarps * 32) attention_simt_kernel(SimtParams 
     }
   }
 
-  T* ob = static_cast<T*>(p.a.out) + size_t(unit) * nt * p.n_q_heads * D;
+  TO* ob = static_cast<TO*>(p.a.out) + size_t(unit) * nt * p.n_q_heads * D;
 #pragma unroll
   for (int r = 0; r < kRows; ++r) {
     const int j = j0 + r;
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kWarps * 32) attention_simt_kernel(SimtParams 
     const float inv = l[r] > 0.f ? 1.f / l[r] : 0.f;
 #pragma unroll
     for (int i = 0; i < D / 32; ++i)
-      ob[(size_t(j) * p.n_q_heads + h) * D + lane + 32 * i] = from_f32<T>(o[r][i] * inv);
+      ob[(size_t(j) * p.n_q_heads + h) * D + lane + 32 * i] = from_f32<TO>(o[r][i] * inv);
     if (p.a.lse && lane == 0)
       p.a.lse[(size_t(unit) * p.n_q_heads + h) * nt + j] = (m[r] + log2f(l[r])) * 0.6931471805599453f;
   }
@@ -204,14 +204,17 @@ int launch_attention_simt(const actqkv_config* cfg, const Batch& b, const AttnAr
   const float scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.f / sqrtf(float(cfg->head_dim));
   p.scale_log2 = scale * 1.4426950408889634f;
   dim3 grid((a.n_tokens + kTileRows - 1) / kTileRows, cfg->n_q_heads, b.units());
-  const bool bf = cfg->dtype == ACTQKV_BF16;
-  if (cfg->head_dim == 128) {
-    if (bf) attention_simt_kernel<__nv_bfloat16, 128><<<grid, kWarps * 32, 0, st>>>(p);
-    else attention_simt_kernel<float, 128><<<grid, kWarps * 32, 0, st>>>(p);
-  } else {
-    if (bf) attention_simt_kernel<__nv_bfloat16, 64><<<grid, kWarps * 32, 0, st>>>(p);
-    else attention_simt_kernel<float, 64><<<grid, kWarps * 32, 0, st>>>(p);
-  }
+  const bool bf = cfg->dtype == ACTQKV_BF16, obf = cfg->out_dtype == ACTQKV_BF16;
+  const int threads = kWarps * 32;
+#define ACTQKV_SIMT_LAUNCH(T, TO, DD) attention_simt_kernel<T, TO, DD><<<grid, threads, 0, st>>>(p)
+#define ACTQKV_SIMT_D(T, TO) \
+  do { if (cfg->head_dim == 128) ACTQKV_SIMT_LAUNCH(T, TO, 128); else ACTQKV_SIMT_LAUNCH(T, TO, 64); } while (0)
+  if (bf && obf) ACTQKV_SIMT_D(__nv_bfloat16, __nv_bfloat16);
+  else if (bf) ACTQKV_SIMT_D(__nv_bfloat16, float);
+  else if (obf) ACTQKV_SIMT_D(float, __nv_bfloat16);
+  else ACTQKV_SIMT_D(float, float);
+#undef ACTQKV_SIMT_D
+#undef ACTQKV_SIMT_LAUNCH
   return launch_status();
 }
 

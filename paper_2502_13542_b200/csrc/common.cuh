@@ -25,6 +25,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int check_config(const actqkv_config* c, const Batch& b) {
   if (!c) return ACTQKV_ERR_NULL;
   if (c->dtype != ACTQKV_F32 && c->dtype != ACTQKV_BF16) return ACTQKV_ERR_DTYPE;
+  if (c->out_dtype != ACTQKV_F32 && c->out_dtype != ACTQKV_BF16) return ACTQKV_ERR_DTYPE;
   if (c->head_dim != 64 && c->head_dim != 128) return ACTQKV_ERR_SHAPE;
   if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_q_heads % c->n_kv_heads) return ACTQKV_ERR_SHAPE;
   if (c->n_q_heads / c->n_kv_heads > 8) return ACTQKV_ERR_SHAPE;

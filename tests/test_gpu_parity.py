@@ -18,16 +18,17 @@ def B():
     return binding
 
 
-def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.0, stop_after=None):
+def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.0, stop_after=None,
+               out_dtype=0):
     """Runs every window of a single-layer workload through RetrievalState.step() and the
     oracle; compares every intermediate.  Returns summary statistics."""
     import torch
-    cfg = B.make_config(spec, beta=beta)
+    cfg = B.make_config(spec, beta=beta, out_dtype=out_dtype)
     n_pages = cfg.n_phys_pages
     pt = wl.shuffled_page_table(spec, spec.context)
     st = B.RetrievalState(cfg, page_table=pt[None, :], keep_phi=True)
     o_run = pu.OracleRunner(spec, beta=beta)
-    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=cfg.torch_dtype, device="cuda")
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=cfg.torch_out_dtype, device="cuda")
     lse = torch.zeros(spec.n_q_heads, spec.window, dtype=torch.float32, device="cuda")
     stats = dict(near=0, worst_att=0.0, worst_att_mean=0.0, worst_rel=0.0, fragile=0)
     last = spec.n_windows if stop_after is None else stop_after
@@ -38,6 +39,7 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
         assert st.host_pos0[0] == p0
         do_att = t in windows_with_attention
         res = o_run.step(q, k, v, attention=do_att)
+        assert int(st.n_cand.item()) == res["n"]
         st.step(pu.to_device(q[None], spec), pu.to_device(k[None], spec), pu.to_device(v[None], spec),
                 out, lse=lse, fused=fused)
         torch.cuda.synchronize()
@@ -46,7 +48,6 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
             continue
         tag = f"{spec.name} window {t}"
         n = res["n"]
-        assert int(st.n_cand.item()) == n
         # step 1: statistics and activation bias
         pu.assert_rel(pu.to_numpy(st.stats_mean[0]), res["zbar"], 1e-3 * np.abs(res["zbar"]).max() + 1e-30, tag + " mean")
         cnt = int(st.stats_count[0, 0].item())
@@ -56,8 +57,8 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
         e1 = pu.assert_phi_like(pu.to_numpy(st.phi_l1[0]).T, res["phi_l1"], tag + " phi_l1")
         e2 = pu.assert_phi_like(pu.to_numpy(st.phi_full[0]), res["phi"], tag + " phi")
         # step 2: probes
-        e3 = pu.assert_phi_like(pu.to_numpy(st.probe_qh[0]), res["probe_qh"], tag + " probe_qh")
-        e4 = pu.assert_phi_like(pu.to_numpy(st.probe_kv[0]), res["probe_kv"], tag + " probe_kv")
+        e3 = pu.assert_probe(pu.to_numpy(st.probe_qh[0]), res["probe_qh"], tag + " probe_qh")
+        e4 = pu.assert_probe(pu.to_numpy(st.probe_kv[0]), res["probe_kv"], tag + " probe_kv")
         # step 3: scores and density
         e5 = 0.0
         if n:
@@ -72,7 +73,8 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
             stats["near"] += nd
         # step 5: attention (only meaningful when the selected sets agree)
         if do_att and nd == 0:
-            mx, mean = pu.assert_attention(pu.to_numpy(out), res["out"], tag + " attention", spec.dtype)
+            check = pu.assert_attention_bf16_out if out_dtype == B.BF16 else pu.assert_attention
+            mx, mean = check(pu.to_numpy(out), res["out"], tag + " attention")
             stats["worst_att"] = max(stats["worst_att"], mx)
             stats["worst_att_mean"] = max(stats["worst_att_mean"], mean)
             pu.assert_rel(pu.to_numpy(lse), res["lse"], 1.0, tag + " lse", tol=2e-3)
@@ -203,7 +205,8 @@ def test_budget_chain_32_layers_matches_oracle(B):
                 assert abs(float(real[l]) - b_real) <= 1e-4 * max(1.0, abs(b_real))
             assert not any(frag)
             assert got_c.tolist() == want_c, (mode_name, step)
-            assert len(set(want_c)) > 2                                   # counts really vary
+            if step > 0 or mode_name == "alg1":
+                assert len(set(want_c)) > 2 and max(want_c) == spec.cap_blocks   # counts vary, cap binds
             for l in range(L):
                 for g in range(Hkv):
                     want, _, _ = orc.select_blocks(s[l, g, :n], want_c[l])
