@@ -1,4 +1,7 @@
 // Helpers of the C ABI and the dispatcher of step 5.
+#include <cstdlib>
+#include <cstring>
+
 #include "common.cuh"
 #include "stages.cuh"
 
@@ -50,5 +53,10 @@ extern "C" int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv
   a.q = q; a.k_win = k_win; a.v_win = v_win; a.k_pages = k_pages; a.v_pages = v_pages;
   a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
   a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
-  return launch_attention_simt(cfg, b, a, reinterpret_cast<cudaStream_t>(stream));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  // ACTQKV_ATTENTION=simt forces the general kernel (debugging aid; the default picks by shape).
+  const char* force = std::getenv("ACTQKV_ATTENTION");
+  const bool simt_only = force && std::strcmp(force, "simt") == 0;
+  if (!simt_only && attention_tc_supported(cfg, n_tokens)) return launch_attention_tc(cfg, b, a, st);
+  return launch_attention_simt(cfg, b, a, st);
 }

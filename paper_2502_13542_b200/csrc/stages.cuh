@@ -40,5 +40,7 @@ struct AttnArgs {
   int n_tokens;
 };
 int launch_attention_simt(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
+bool attention_tc_supported(const actqkv_config* cfg, int n_tokens);
+int launch_attention_tc(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 
 }  // namespace actqkv
