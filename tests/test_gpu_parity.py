@@ -263,3 +263,47 @@ def test_edge_cases_and_errors(B):
                                     f"ragged {nt}") == 0
         pu.assert_attention(pu.to_numpy(o), res["out"], f"ragged step of {nt} tokens")
     assert int(st4.status.item()) == 0
+
+
+@pytest.mark.parametrize("target", [1, 3])
+def test_tc_attention_repeatable_and_matches_general_kernel(B, monkeypatch, target):
+    """The tensor-core attention is run many times on the same state: every run must give the
+    same bits (no timing dependence), and agree with the general fp32 kernel.  Window 1 gives
+    the shortest key-tile loops (5 to 8 tiles), window 3 longer ones."""
+    import torch
+    spec = wl.llama3_8b_layer().replace(context=4096)
+    cfg = B.make_config(spec, out_dtype=B.F32)
+    st = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :])
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    for t in range(target + 1):
+        q = pu.to_device(wl.gen_q(spec, 0, t)[None], spec)
+        k, v = wl.gen_kv(spec, 0, t)
+        k, v = pu.to_device(k[None], spec), pu.to_device(v[None], spec)
+        if t < target:
+            st.step(q, k, v, out)
+    # state now stands at the target window; score/select once, then attention repeatedly
+    B.bias_probe(cfg, st.batch, q, spec.window, st.stats_count, st.stats_mean, st.stats_m2, st.phi_l1, None,
+                 st.probe_qh, st.probe_kv, st.status)
+    B.score_select(cfg, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, st.budget_state, st.scores,
+                   st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
+
+    def attend(dst):
+        B.retrieval_attention(cfg, st.batch, q, k, v, spec.window, st.k_pages, st.v_pages, st.page_table, st.pos0,
+                              st.sel_idx, st.sel_count, dst, None, st.status)
+    monkeypatch.setenv("ACTQKV_ATTENTION", "simt")
+    gen = torch.zeros_like(out)
+    attend(gen)
+    torch.cuda.synchronize()
+    monkeypatch.delenv("ACTQKV_ATTENTION")
+    outs = [torch.zeros_like(out) for _ in range(8)]
+    ref = None
+    for rep in range(60):
+        for o in outs:
+            attend(o)
+        torch.cuda.synchronize()
+        if ref is None:
+            ref = outs[0].clone()
+            assert (gen - ref).abs().max().item() < 2e-3
+        for o in outs:
+            assert torch.equal(o, ref), f"run {rep}: tensor-core attention not repeatable"
+    assert int(st.status.item()) == 0
