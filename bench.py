@@ -201,11 +201,16 @@ def run_ours(args):
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
+    if args.profile_region:
+        torch.cuda.profiler.start()          # cudaProfilerStart: lets a profiler capture the timed region only
     e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
         one_step(args.warmup + i)
     e1.record()
+    if args.profile_region:
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
     sampler.sample()
     barrier()
     clocks = sampler.stop()
@@ -376,6 +381,8 @@ def main():
     ap.add_argument("--copies", type=int, default=8)
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-region", action="store_true",
+                    help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
