@@ -9,15 +9,21 @@
 // The block -> page indirection (sel_idx, page_table) is resolved by the producer warp, one
 // lane per box.  The window's own keys / values come from k_win / v_win with one box per half.
 //
-//   warp 0      TMA producer (3-stage ring of K+V tiles)
-//   warp 1      tcgen05.mma issuer (one lane), owns the TMEM allocation
-//   warps 2-5   softmax: one thread per query row (TMEM lane), running max / sum in base 2,
-//               P written back to TMEM as two bf16 terms (hi, lo) over the S columns, O rescaled in TMEM only
-//               when a row's max grew by more than 2^8 (lazy rescale), epilogue.
+// Three warpgroups:
+//   warp 0        TMA producer (3-stage ring of K+V tiles)
+//   warp 1        tcgen05.mma issuer (one lane), owns the TMEM allocation
+//   warps 4-7     softmax of the even key tiles, accumulator O0
+//   warps 8-11    softmax of the odd key tiles, accumulator O1
+// Each softmax thread owns one query row (= TMEM lane): running max / sum in base 2, P written
+// back over the S columns as two bf16 terms (hi + lo), its O rescaled in TMEM only when the
+// row's max grew by more than 2^8 (lazy rescale).  The two warpgroups keep independent
+// (max, sum, O) triples, so the tensor pipe works on one tile's P V while the other tile's
+// softmax runs; the epilogue merges the two partial results per row.
 //
-// TMEM columns: S0/P0 [0,128)  S1/P1 [128,256)  O [256,384)  (512 allocated).
+// TMEM columns: S0/P0 [0,128)  S1/P1 [128,256)  O0 [256,384)  O1 [384,512).
 // S = Q K^T uses both operands from shared memory (K-major, SW128); O += P V takes P from
 // TMEM and V from shared memory as an MN-major operand (the V tile is [keys x channels]).
+// P of keys [32c, 32c+32) of a tile lives in columns [32c, 32c+16) (hi) and [32c+16, 32c+32) (lo).
 // Every wait on an mbarrier is bounded; on expiry the CTA flags ACTQKV_DEV_TIMEOUT, stops
 // issuing work, drains and frees its TMEM.
 #include <cuda.h>
@@ -31,7 +37,7 @@ namespace {
 
 constexpr int kBM = 128, kBN = 128, kD = 128;
 constexpr int kStages = 3;
-constexpr int kThreads = 192;
+constexpr int kThreads = 384;                           // 3 warpgroups
 constexpr uint32_t kSubTileBytes = 128 * 128;            // [128 rows x 64 bf16], 16 KiB
 constexpr uint32_t kTileBytes = 2 * kSubTileBytes;       // 32 KiB: one K or V or Q tile
 constexpr uint32_t kStageBytes = 2 * kTileBytes;         // K + V
@@ -147,7 +153,6 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),      \
         "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])                                           \
       : "memory")
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
@@ -172,6 +177,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // ---------------------------------------------------------------- kernel
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Barrier among the 256 softmax threads only (hardware barrier 1; barrier 0 is __syncthreads).
+__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kw,
                     const __grid_constant__ CUtensorMap tm_vw, const __grid_constant__ CUtensorMap tm_kp,
@@ -188,10 +201,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   auto bar_empty = [&](int s) { return bars + 8u * (1 + 2 * kStages + s); };
   auto bar_sfull = [&](int b) { return bars + 8u * (1 + 3 * kStages + b); };
   auto bar_pfull = [&](int b) { return bars + 8u * (3 + 3 * kStages + b); };
-  const uint32_t bar_pvdone = bars + 8u * (5 + 3 * kStages);
-  unsigned char* bars_generic = smem_raw + (bars - smem_u32(smem_raw));
+  const uint32_t bar_done = bars + 8u * (5 + 3 * kStages);
+  unsigned char* base_generic = smem_raw + (base - smem_u32(smem_raw));
+  unsigned char* bars_generic = base_generic + kSmemData;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * (6 + 3 * kStages));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * (6 + 3 * kStages) + 8);
+  // after the last MMA has completed the Q tile is dead: its first 2 KiB carry the two
+  // warpgroups' (max, sum) pairs to the merge
+  float2* merge_ml = reinterpret_cast<float2*>(base_generic);
 
   const int mt = blockIdx.x, h = blockIdx.y, unit = blockIdx.z;
   const int g = h / p.group, seq = unit / p.n_layers, layer_local = unit - seq * p.n_layers;
@@ -222,7 +239,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(bar_q, 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_vfull(s), 1); mbar_init(bar_empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 128); }
-    mbar_init(bar_pvdone, 1);
+    mbar_init(bar_done, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -240,132 +257,142 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     return;
   }
 
-  if (warp == 0) {
-    // =========================== TMA producer ===========================
-    const int32_t* sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
-    const int32_t* pt = p.a.page_table + size_t(seq) * p.max_pages;
-    const int page_oob = p.n_layers * p.n_phys_pages;              // beyond the tensor: zero fill
-    if (lane == 0) {
-      mbar_expect_tx(bar_q, kTileBytes);
-      tma_load_3d(q_smem, &tm_q, bar_q, 0, h, unit * nt + mt * kBM);
-      tma_load_3d(q_smem + kSubTileBytes, &tm_q, bar_q, 64, h, unit * nt + mt * kBM);
-    }
-    bool ok = true;
-    int issued = 0;
-    for (int j = 0; j < n_tiles && ok; ++j) {
-      const int s = j % kStages, it = j / kStages;
-      if (it > 0) ok = mbar_wait(bar_empty(s), (it - 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      const uint32_t sbase = stage0 + s * kStageBytes;
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    if (warp == 0) {
+      // =========================== TMA producer ===========================
+      const int32_t* sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
+      const int32_t* pt = p.a.page_table + size_t(seq) * p.max_pages;
+      const int page_oob = p.n_layers * p.n_phys_pages;              // beyond the tensor: zero fill
       if (lane == 0) {
-        mbar_expect_tx(bar_kfull(s), kTileBytes);
-        mbar_expect_tx(bar_vfull(s), kTileBytes);
+        mbar_expect_tx(bar_q, kTileBytes);
+        tma_load_3d(q_smem, &tm_q, bar_q, 0, h, unit * nt + mt * kBM);
+        tma_load_3d(q_smem + kSubTileBytes, &tm_q, bar_q, 64, h, unit * nt + mt * kBM);
       }
-      __syncwarp();
-      if (j < past_tiles) {
-        const int is_v = lane >> 4, half = (lane >> 3) & 1, slot = lane & 7;
-        const int gi = j * 8 + slot;
-        int page = page_oob;
-        if (gi < g_past) {
-          int64_t lp;
-          if (gi < g_init) {
-            lp = gi;
-          } else if (gi < g_init + g_sel) {
-            const int r = gi - g_init;
-            const int blk = sel[r / gpb];
-            lp = (blk >= 0 && blk < geo.n_cand) ? (int64_t(p.n_init) + int64_t(blk) * p.block) / 16 + r % gpb : -1;
-            if (lp < 0 && half == 0 && is_v == 0) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
-          } else {
-            lp = geo.local_start / 16 + (gi - g_init - g_sel);
-          }
-          if (lp >= 0) {
-            const int phys = lp < p.max_pages ? pt[lp] : -1;
-            if (phys < 0 || phys >= p.n_phys_pages) {
-              if (half == 0 && is_v == 0) set_status(p.a.status, ACTQKV_DEV_BAD_PAGE);
+      bool ok = true;
+      int issued = 0;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int s = j % kStages, it = j / kStages;
+        if (it > 0) ok = mbar_wait(bar_empty(s), (it - 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t sbase = stage0 + s * kStageBytes;
+        if (lane == 0) {
+          mbar_expect_tx(bar_kfull(s), kTileBytes);
+          mbar_expect_tx(bar_vfull(s), kTileBytes);
+        }
+        __syncwarp();
+        if (j < past_tiles) {
+          const int is_v = lane >> 4, half = (lane >> 3) & 1, slot = lane & 7;
+          const int gi = j * 8 + slot;
+          int page = page_oob;
+          if (gi < g_past) {
+            int64_t lp;
+            if (gi < g_init) {
+              lp = gi;
+            } else if (gi < g_init + g_sel) {
+              const int r = gi - g_init;
+              const int blk = sel[r / gpb];
+              lp = (blk >= 0 && blk < geo.n_cand) ? (int64_t(p.n_init) + int64_t(blk) * p.block) / 16 + r % gpb : -1;
+              if (lp < 0 && half == 0 && is_v == 0) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
             } else {
-              page = layer_local * p.n_phys_pages + phys;
+              lp = geo.local_start / 16 + (gi - g_init - g_sel);
+            }
+            if (lp >= 0) {
+              const int phys = lp < p.max_pages ? pt[lp] : -1;
+              if (phys < 0 || phys >= p.n_phys_pages) {
+                if (half == 0 && is_v == 0) set_status(p.a.status, ACTQKV_DEV_BAD_PAGE);
+              } else {
+                page = layer_local * p.n_phys_pages + phys;
+              }
             }
           }
+          const uint32_t dst = sbase + is_v * kTileBytes + half * kSubTileBytes + slot * 2048u;
+          tma_load_4d(dst, is_v ? &tm_vp : &tm_kp, is_v ? bar_vfull(s) : bar_kfull(s), half * 64, 0, g, page);
+        } else if (lane < 4) {
+          const int is_v = lane >> 1, half = lane & 1;
+          const int kt = j - past_tiles;
+          const uint32_t dst = sbase + is_v * kTileBytes + half * kSubTileBytes;
+          tma_load_3d(dst, is_v ? &tm_vw : &tm_kw, is_v ? bar_vfull(s) : bar_kfull(s), half * 64, g,
+                      unit * nt + kt * kBN);
         }
-        const uint32_t dst = sbase + is_v * kTileBytes + half * kSubTileBytes + slot * 2048u;
-        tma_load_4d(dst, is_v ? &tm_vp : &tm_kp, is_v ? bar_vfull(s) : bar_kfull(s), half * 64, 0, g, page);
-      } else if (lane < 4) {
-        const int is_v = lane >> 1, half = lane & 1;
-        const int kt = j - past_tiles;
-        const uint32_t dst = sbase + is_v * kTileBytes + half * kSubTileBytes;
-        tma_load_3d(dst, is_v ? &tm_vw : &tm_kw, is_v ? bar_vfull(s) : bar_kfull(s), half * 64, g,
-                    unit * nt + kt * kBN);
+        issued = j + 1;
       }
-      issued = j + 1;
-    }
-    // drain: every issued copy must have landed before the CTA may exit on the abort path
-    if (!ok) {
-      for (int j = max(0, issued - kStages); j < issued; ++j) {
-        const int s = j % kStages, par = (j / kStages) & 1;
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_kfull(s), par); ++i) {}
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_vfull(s), par); ++i) {}
+      // drain: every issued copy must have landed before the CTA may exit on the abort path
+      if (!ok) {
+        for (int j = max(0, issued - kStages); j < issued; ++j) {
+          const int s = j % kStages, par = (j / kStages) & 1;
+          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_kfull(s), par); ++i) {}
+          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_vfull(s), par); ++i) {}
+        }
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
       }
-      for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
-    }
-  } else if (warp == 1) {
-    // =========================== MMA issuer ===========================
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc(false);
-      constexpr uint32_t idesc_pv = make_idesc(true);
-      const uint32_t tmem_o = tmem + 256;
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
-      auto issue_pv = [&](int i) {
-        const int s = i % kStages;
-        ok = ok && mbar_wait(bar_vfull(s), (i / kStages) & 1, abort_flag);
-        ok = ok && mbar_wait(bar_pfull(i & 1), (i >> 1) & 1, abort_flag);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t vbase = stage0 + s * kStageBytes + kTileBytes;
-        const uint32_t p_tmem = tmem + (i & 1) * 128;
+    } else if (warp == 1) {
+      // =========================== MMA issuer ===========================
+      // Issue order QK(0), QK(1), PV(0), QK(2), PV(1), ...: the tensor pipe executes in issue
+      // order, so QK(j+2) cannot overwrite S/P buffer j&1 before PV(j) has read P(j), and a
+      // completed QK(j) implies a completed PV(j-2).
+      if (lane == 0) {
+        constexpr uint32_t idesc_qk = make_idesc(false);
+        constexpr uint32_t idesc_pv = make_idesc(true);
+        bool ok = mbar_wait(bar_q, 0, abort_flag);
+        auto issue_pv = [&](int i) {
+          const int s = i % kStages, b = i & 1;
+          ok = ok && mbar_wait(bar_vfull(s), (i / kStages) & 1, abort_flag);
+          ok = ok && mbar_wait(bar_pfull(b), (i >> 1) & 1, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
+          const uint32_t vbase = stage0 + s * kStageBytes + kTileBytes;
+          const uint32_t p_tmem = tmem + b * 128;
+          const uint32_t o_tmem = tmem + 256 + b * 128;
 #pragma unroll
-        for (int k = 0; k < kBN / 16; ++k) {
-          // 16 keys per step: A advances 8 packed columns, B advances 16 rows of 128 bytes;
-          // the hi and lo halves of P (columns [0,64) and [64,128)) multiply the same V rows.
-          const uint64_t bdesc = make_desc(vbase + k * 2048u, kSubTileBytes, 1024u);
-          mma_ts(tmem_o, p_tmem + k * 8, bdesc, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
-          mma_ts(tmem_o, p_tmem + 64 + k * 8, bdesc, idesc_pv, 1u);
-        }
-        tc_commit(bar_empty(s));
-        tc_commit(bar_pvdone);
-      };
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j % kStages;
-        ok = mbar_wait(bar_kfull(s), (j / kStages) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t kbase = stage0 + s * kStageBytes;
+          for (int k = 0; k < kBN / 16; ++k) {
+            // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
+            // term, then the 8 columns of the lo term of the same keys against the same V rows.
+            const uint64_t bdesc = make_desc(vbase + k * 2048u, kSubTileBytes, 1024u);
+            const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
+            mma_ts(o_tmem, pa, bdesc, idesc_pv, (i >= 2 || k > 0) ? 1u : 0u);
+            mma_ts(o_tmem, pa + 16, bdesc, idesc_pv, 1u);
+          }
+          tc_commit(bar_empty(s));
+        };
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const int s = j % kStages;
+          ok = mbar_wait(bar_kfull(s), (j / kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t kbase = stage0 + s * kStageBytes;
 #pragma unroll
-        for (int k = 0; k < kD / 16; ++k) {
-          const uint32_t off = (k >> 2) * kSubTileBytes + (k & 3) * 32u;
-          const uint64_t adesc = make_desc(q_smem + off, 16u, 1024u);
-          const uint64_t bdesc = make_desc(kbase + off, 16u, 1024u);
-          mma_ss(tmem + (j & 1) * 128, adesc, bdesc, idesc_qk, k > 0 ? 1u : 0u);
+          for (int k = 0; k < kD / 16; ++k) {
+            const uint32_t off = (k >> 2) * kSubTileBytes + (k & 3) * 32u;
+            const uint64_t adesc = make_desc(q_smem + off, 16u, 1024u);
+            const uint64_t bdesc = make_desc(kbase + off, 16u, 1024u);
+            mma_ss(tmem + (j & 1) * 128, adesc, bdesc, idesc_qk, k > 0 ? 1u : 0u);
+          }
+          tc_commit(bar_sfull(j & 1));
+          if (j >= 1) issue_pv(j - 1);
         }
-        tc_commit(bar_sfull(j & 1));
-        if (j >= 1) issue_pv(j - 1);
+        if (ok) issue_pv(n_tiles - 1);
+        if (ok) tc_commit(bar_done);
       }
-      if (ok) issue_pv(n_tiles - 1);
+      __syncwarp();
     }
-    __syncwarp();
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     // =========================== softmax / epilogue ===========================
+    const int b = (warp >> 2) - 1;                        // 0: even tiles, 1: odd tiles
     const int q4 = warp & 3;                              // TMEM lane quadrant of this warp
     const int row = q4 * 32 + lane;                       // query row inside the tile
     const uint32_t lane_addr = uint32_t(q4 * 32) << 16;
+    const uint32_t s_addr = tmem + lane_addr + b * 128;
+    const uint32_t o_addr = tmem + lane_addr + 256 + b * 128;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      ok = ok && mbar_wait(bar_sfull(j & 1), (j >> 1) & 1, abort_flag);
+    for (int j = b, kk = 0; j < n_tiles; j += 2, ++kk) {
+      ok = ok && mbar_wait(bar_sfull(b), kk & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t s_addr = tmem + lane_addr + (j & 1) * 128;
       uint32_t sr[128];
       TMEM_LD128_WAIT(s_addr, sr);
       // key-validity limit: ragged last past tile, or the causal diagonal of the last tile
@@ -377,31 +404,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (masked) {
 #pragma unroll
         for (int i = 0; i < 128; ++i) {
-          float x = __uint_as_float(sr[i]) * p.scale_log2;
-          x = i < limit ? x : -INFINITY;
+          const float x = i < limit ? __uint_as_float(sr[i]) : -INFINITY;
           sr[i] = __float_as_uint(x);
           mx = fmaxf(mx, x);
         }
       } else {
+        float mx2 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 128; ++i) {
-          const float x = __uint_as_float(sr[i]) * p.scale_log2;
-          sr[i] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
+        for (int i = 0; i < 128; i += 2) {
+          mx = fmaxf(mx, __uint_as_float(sr[i]));
+          mx2 = fmaxf(mx2, __uint_as_float(sr[i + 1]));
         }
+        mx = fmaxf(mx, mx2);
       }
-      const float m_new = fmaxf(m_used, mx);
+      const float m_new = fmaxf(m_used, mx * p.scale_log2);
       const bool grow = m_new - m_used > kRescaleThreshold;     // also true for the first tile
-      if (j == 0) {
+      if (kk == 0) {
         m_used = m_new;
       } else if (__any_sync(0xffffffffu, grow)) {
-        ok = mbar_wait(bar_pvdone, (j - 1) & 1, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
-        const float f = grow ? exp2f(m_used - m_new) : 1.f;
+        // S(j) complete implies PV(j-2) complete: this warpgroup's O is quiescent until it
+        // publishes P(j)
+        const float f = grow ? ex2(m_used - m_new) : 1.f;
         if (grow) { m_used = m_new; l *= f; }
-        const uint32_t o_addr = tmem + lane_addr + 256;
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
           uint32_t orr[32];
@@ -410,70 +434,81 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
           TMEM_ST32(o_addr + cc * 32, orr);
         }
-        tmem_wait_st();
       }
       // P = exp2(x - m) split into two bf16 terms (hi + lo): with outlier value channels a
       // single bf16 P (8 significant bits) would cost up to |v| * 2^-9 of absolute error.
-      float sum = 0.f;
-      uint32_t pk[64], pl[64];
-#pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float e0 = exp2f(__uint_as_float(sr[2 * i]) - m_used);
-        const float e1 = exp2f(__uint_as_float(sr[2 * i + 1]) - m_used);
-        sum += e0 + e1;
-        const uint32_t hi = pack_bf16(e0, e1);
-        pk[i] = hi;
-        pl[i] = pack_bf16(e0 - __uint_as_float(hi << 16), e1 - __uint_as_float(hi & 0xFFFF0000u));
-      }
-      l += sum;
-      TMEM_ST32(s_addr, (pk + 0));
-      TMEM_ST32(s_addr + 32, (pk + 32));
-      TMEM_ST32(s_addr + 64, (pl + 0));
-      TMEM_ST32(s_addr + 96, (pl + 32));
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_pfull(j & 1));
-    }
-    // ---- epilogue: O / l -> global.  A parity wait can only tell the phase in progress from the
-    // one before it, and after the last S tile the barrier may still be in phase n_tiles - 2 (this
-    // warp may not have waited on it for many tiles): pass that phase first, then the last one.
-    if (ok && n_tiles >= 2) ok = mbar_wait(bar_pvdone, (n_tiles - 2) & 1, abort_flag);
-    if (ok) ok = mbar_wait(bar_pvdone, (n_tiles - 1) & 1, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-      tc_fence_after();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      const size_t tok = size_t(unit) * nt + size_t(mt) * kBM + row;
-      const uint32_t o_addr = tmem + lane_addr + 256;
+      const float neg_m = -m_used;
+      float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
-        uint32_t orr[32];
-        TMEM_LD32_WAIT(o_addr + cc * 32, orr);
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float e0 = ex2(fmaf(__uint_as_float(sr[32 * cc + 2 * i]), p.scale_log2, neg_m));
+          const float e1 = ex2(fmaf(__uint_as_float(sr[32 * cc + 2 * i + 1]), p.scale_log2, neg_m));
+          sum0 += e0;
+          sum1 += e1;
+          const uint32_t hi = pack_bf16(e0, e1);
+          pk[i] = hi;
+          pk[16 + i] = pack_bf16(e0 - __uint_as_float(hi << 16), e1 - __uint_as_float(hi & 0xFFFF0000u));
+        }
+        TMEM_ST32(s_addr + cc * 32, pk);
+      }
+      l += sum0 + sum1;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_pfull(b));
+    }
+    // ---- merge of the two warpgroups' partial results and epilogue
+    ok = ok && mbar_wait(bar_done, 0, abort_flag);
+    if (ok) merge_ml[b * 128 + row] = make_float2(m_used, l);
+    softmax_sync();
+    if (*abort_flag == 0) {
+      tc_fence_after();
+      const float2 a0 = merge_ml[row], a1 = merge_ml[128 + row];
+      const float m = fmaxf(a0.x, a1.x);
+      float f0 = a0.y > 0.f ? ex2(a0.x - m) : 0.f;
+      float f1 = a1.y > 0.f ? ex2(a1.x - m) : 0.f;
+      const float lsum = a0.y * f0 + a1.y * f1;
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      f0 *= inv;
+      f1 *= inv;
+      const bool use1 = f1 != 0.f;                          // O1 was never written when the CTA has one tile
+      const size_t tok = size_t(unit) * nt + size_t(mt) * kBM + row;
+      const uint32_t o0 = tmem + lane_addr + 256, o1 = tmem + lane_addr + 384;
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        const int col = b * 64 + cc * 32;                   // this warpgroup's half of the channels
+        uint32_t r0[32], r1[32];
+        TMEM_LD32_WAIT(o0 + col, r0);
+        TMEM_LD32_WAIT(o1 + col, r1);
+        float o[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float x1 = use1 ? __uint_as_float(r1[i]) * f1 : 0.f;
+          o[i] = fmaf(__uint_as_float(r0[i]), f0, x1);
+        }
         if (p.out_bf16) {
-          __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + cc * 32;
+          __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             uint4 v;
-            v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
-            v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
-            v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
-            v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+            v.x = pack_bf16(o[8 * i + 0], o[8 * i + 1]);
+            v.y = pack_bf16(o[8 * i + 2], o[8 * i + 3]);
+            v.z = pack_bf16(o[8 * i + 4], o[8 * i + 5]);
+            v.w = pack_bf16(o[8 * i + 6], o[8 * i + 7]);
             *reinterpret_cast<uint4*>(ob + 8 * i) = v;
           }
         } else {
-          float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + cc * 32;
+          float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float4 v;
-            v.x = __uint_as_float(orr[4 * i + 0]) * inv; v.y = __uint_as_float(orr[4 * i + 1]) * inv;
-            v.z = __uint_as_float(orr[4 * i + 2]) * inv; v.w = __uint_as_float(orr[4 * i + 3]) * inv;
-            *reinterpret_cast<float4*>(of + 4 * i) = v;
-          }
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<float4*>(of + 4 * i) = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
         }
       }
-      if (p.a.lse)
+      if (p.a.lse && b == 0)
         p.a.lse[(size_t(unit) * p.n_q_heads + h) * nt + size_t(mt) * kBM + row] =
-            (m_used + log2f(l)) * 0.6931471805599453f;
+            (m + log2f(lsum)) * 0.6931471805599453f;
     }
   }
 
