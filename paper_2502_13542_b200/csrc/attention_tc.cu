@@ -6,24 +6,26 @@
 // Key tiles of 128 keys are gathered page by page: each 16-token page is one TMA box of
 // 16 rows x 128 bytes per 64-channel half, written with the 128-byte swizzle the MMA
 // descriptors expect, so a [128 x 64] operand sub-tile is 8 boxes stacked in shared memory.
-// The block -> page indirection (sel_idx, page_table) is resolved by the producer warp, one
+// The block -> page indirection (sel_idx, page_table) is resolved by the producer warps, one
 // lane per box.  The window's own keys / values come from k_win / v_win with one box per half.
 //
-// Three warpgroups:
-//   warp 0        TMA producer (3-stage ring of K+V tiles)
+// Three warpgroups (384 threads):
+//   warp 0        TMA producer of the K tiles (ring of 3) and of the Q tile
 //   warp 1        tcgen05.mma issuer (one lane), owns the TMEM allocation
-//   warps 4-7     softmax of the even key tiles, accumulator O0
-//   warps 8-11    softmax of the odd key tiles, accumulator O1
-// Each softmax thread owns one query row (= TMEM lane): running max / sum in base 2, P written
-// back over the S columns as two bf16 terms (hi + lo), its O rescaled in TMEM only when the
-// row's max grew by more than 2^8 (lazy rescale).  The two warpgroups keep independent
-// (max, sum, O) triples, so the tensor pipe works on one tile's P V while the other tile's
-// softmax runs; the epilogue merges the two partial results per row.
+//   warp 2        TMA producer of the V tiles (ring of 3, released separately from K)
+//   warps 4-7     softmax, key columns [0, 64) of every tile (packed f32x2 arithmetic)
+//   warps 8-11    softmax, key columns [64, 128) of every tile
+// A query row (= TMEM lane) is shared by two softmax threads, one per column half; they
+// exchange their half-row maxima through shared memory once per tile.  Running max / sum are
+// kept in base 2; P is written back over the S columns as two bf16 terms (hi + lo); O is
+// rescaled in TMEM only when a row's max grew by more than 2^8 (lazy rescale).
 //
-// TMEM columns: S0/P0 [0,128)  S1/P1 [128,256)  O0 [256,384)  O1 [384,512).
+// TMEM columns: S/P buffers 0..2 at [0,128) [128,256) [256,384), O at [384,512).
 // S = Q K^T uses both operands from shared memory (K-major, SW128); O += P V takes P from
 // TMEM and V from shared memory as an MN-major operand (the V tile is [keys x channels]).
 // P of keys [32c, 32c+32) of a tile lives in columns [32c, 32c+16) (hi) and [32c+16, 32c+32) (lo).
+// The tensor pipe executes in issue order QK(0) QK(1) | QK(j+2) PV(j) ..., so S(j+2) is computed
+// while the softmax of tile j+1 runs and QK(j+3) cannot overwrite buffer j%3 before PV(j) read it.
 // Every wait on an mbarrier is bounded; on expiry the CTA flags ACTQKV_DEV_TIMEOUT, stops
 // issuing work, drains and frees its TMEM.
 #include <cuda.h>
@@ -36,13 +38,20 @@ using namespace actqkv;
 namespace {
 
 constexpr int kBM = 128, kBN = 128, kD = 128;
-constexpr int kStages = 3;
-constexpr int kThreads = 384;                           // 3 warpgroups
+constexpr int kRing = 3;                                 // K tiles in flight, and V tiles in flight
+constexpr int kSBuf = 3;                                 // S/P buffers in TMEM
+constexpr int kPvRing = 4;                               // barriers that count completed P V products
+constexpr int kThreads = 384;                            // 3 warpgroups
 constexpr uint32_t kSubTileBytes = 128 * 128;            // [128 rows x 64 bf16], 16 KiB
 constexpr uint32_t kTileBytes = 2 * kSubTileBytes;       // 32 KiB: one K or V or Q tile
-constexpr uint32_t kStageBytes = 2 * kTileBytes;         // K + V
-constexpr uint32_t kSmemData = kTileBytes + kStages * kStageBytes;
-constexpr uint32_t kSmemBytes = kSmemData + 1024 /*align*/ + 256 /*barriers*/;
+constexpr uint32_t kSmemTiles = (1 + 2 * kRing) * kTileBytes;
+constexpr int kNumBars = 1 + 4 * kRing + 2 * kSBuf + kPvRing + 1;
+constexpr uint32_t kBarBytes = 256;                      // barriers, TMEM slot, abort flag
+constexpr uint32_t kXchgBytes = 2 * 2 * 128 * 4;         // [tile parity][column half][row] floats
+constexpr uint32_t kSmemNeeded = kSmemTiles + kBarBytes + kXchgBytes;
+constexpr uint32_t kSmemBytes = 227 * 1024;              // everything an SM offers one CTA
+static_assert(8 * kNumBars + 16 <= kBarBytes, "barrier area too small");
+static_assert(kSmemNeeded <= kSmemBytes, "shared memory budget");
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
 
@@ -114,44 +123,70 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
-#define TMEM_LD32(taddr, r)                                                                      \
-  asm volatile(                                                                                  \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,"  \
-      "%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"         \
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),      \
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),  \
-        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),            \
-        "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),            \
-        "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])             \
-      : "r"(taddr))
-// Four 32-column loads and the wait in ONE asm statement: no consumer of the registers can be
-// scheduled ahead of tcgen05.wait::ld.
-#define TMEM_LD128_WAIT(taddr, r)                                                              \
-  asm volatile(                                                                                \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%128];\n\t"                            \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%129];\n\t"                            \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%64,%65,%66,%67,%68,%69,%70,%71,%72,%73,%74,%75,%76,%77,%78,%79,%80,%81,%82,%83,%84,%85,%86,%87,%88,%89,%90,%91,%92,%93,%94,%95}, [%130];\n\t"                            \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%96,%97,%98,%99,%100,%101,%102,%103,%104,%105,%106,%107,%108,%109,%110,%111,%112,%113,%114,%115,%116,%117,%118,%119,%120,%121,%122,%123,%124,%125,%126,%127}, [%131];\n\t"                            \
-      "tcgen05.wait::ld.sync.aligned;"                                                         \
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95]), "=r"(r[96]), "=r"(r[97]), "=r"(r[98]), "=r"(r[99]), "=r"(r[100]), "=r"(r[101]), "=r"(r[102]), "=r"(r[103]), "=r"(r[104]), "=r"(r[105]), "=r"(r[106]), "=r"(r[107]), "=r"(r[108]), "=r"(r[109]), "=r"(r[110]), "=r"(r[111]), "=r"(r[112]), "=r"(r[113]), "=r"(r[114]), "=r"(r[115]), "=r"(r[116]), "=r"(r[117]), "=r"(r[118]), "=r"(r[119]), "=r"(r[120]), "=r"(r[121]), "=r"(r[122]), "=r"(r[123]), "=r"(r[124]), "=r"(r[125]), "=r"(r[126]), "=r"(r[127])                                                                                     \
-      : "r"(taddr), "r"((taddr) + 32), "r"((taddr) + 64), "r"((taddr) + 96)                    \
+// TMEM loads come with their wait in ONE asm statement, so that no consumer of the registers
+// can be scheduled ahead of tcgen05.wait::ld.
+#define TMEM_LD64_WAIT(taddr, r) \
+  asm volatile( \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%64];\n\t" \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%65];\n\t" \
+      "tcgen05.wait::ld.sync.aligned;" \
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]) \
+      : "r"(taddr), "r"((taddr) + 32) \
       : "memory")
-#define TMEM_LD32_WAIT(taddr, r)                                                               \
-  asm volatile(                                                                                \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"                             \
-      "tcgen05.wait::ld.sync.aligned;"                                                         \
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])                                                                                     \
-      : "r"(taddr)                                                                             \
+#define TMEM_LD32_WAIT(taddr, r) \
+  asm volatile( \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t" \
+      "tcgen05.wait::ld.sync.aligned;" \
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]) \
+      : "r"(taddr) \
       : "memory")
-#define TMEM_ST32(taddr, r)                                                                      \
-  asm volatile(                                                                                  \
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,"   \
-      "%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"        \
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), \
-        "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),         \
-        "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),      \
-        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),      \
-        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])                                           \
+#define TMEM_ST32(taddr, r) \
+  asm volatile( \
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" \
+      :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) \
+      : "memory")
+// 64 columns as 32 register pairs (column 2i in the low half of r[i]), for the packed f32x2 pipe.
+#define TMEM_LD64P_WAIT(taddr, r) \
+  asm volatile( \
+      "{\n\t.reg .b32 t<64>;\n\t" \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t0,t1,t2,t3,t4,t5,t6,t7,t8,t9,t10,t11,t12,t13,t14,t15,t16,t17,t18,t19,t20,t21,t22,t23,t24,t25,t26,t27,t28,t29,t30,t31}, [%32];\n\t" \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t32,t33,t34,t35,t36,t37,t38,t39,t40,t41,t42,t43,t44,t45,t46,t47,t48,t49,t50,t51,t52,t53,t54,t55,t56,t57,t58,t59,t60,t61,t62,t63}, [%33];\n\t" \
+      "tcgen05.wait::ld.sync.aligned;\n\t" \
+      "mov.b64 %0, {t0, t1};\n\t" \
+      "mov.b64 %1, {t2, t3};\n\t" \
+      "mov.b64 %2, {t4, t5};\n\t" \
+      "mov.b64 %3, {t6, t7};\n\t" \
+      "mov.b64 %4, {t8, t9};\n\t" \
+      "mov.b64 %5, {t10, t11};\n\t" \
+      "mov.b64 %6, {t12, t13};\n\t" \
+      "mov.b64 %7, {t14, t15};\n\t" \
+      "mov.b64 %8, {t16, t17};\n\t" \
+      "mov.b64 %9, {t18, t19};\n\t" \
+      "mov.b64 %10, {t20, t21};\n\t" \
+      "mov.b64 %11, {t22, t23};\n\t" \
+      "mov.b64 %12, {t24, t25};\n\t" \
+      "mov.b64 %13, {t26, t27};\n\t" \
+      "mov.b64 %14, {t28, t29};\n\t" \
+      "mov.b64 %15, {t30, t31};\n\t" \
+      "mov.b64 %16, {t32, t33};\n\t" \
+      "mov.b64 %17, {t34, t35};\n\t" \
+      "mov.b64 %18, {t36, t37};\n\t" \
+      "mov.b64 %19, {t38, t39};\n\t" \
+      "mov.b64 %20, {t40, t41};\n\t" \
+      "mov.b64 %21, {t42, t43};\n\t" \
+      "mov.b64 %22, {t44, t45};\n\t" \
+      "mov.b64 %23, {t46, t47};\n\t" \
+      "mov.b64 %24, {t48, t49};\n\t" \
+      "mov.b64 %25, {t50, t51};\n\t" \
+      "mov.b64 %26, {t52, t53};\n\t" \
+      "mov.b64 %27, {t54, t55};\n\t" \
+      "mov.b64 %28, {t56, t57};\n\t" \
+      "mov.b64 %29, {t58, t59};\n\t" \
+      "mov.b64 %30, {t60, t61};\n\t" \
+      "mov.b64 %31, {t62, t63};\n\t" \
+      "}" \
+      : "=l"(r[0]), "=l"(r[1]), "=l"(r[2]), "=l"(r[3]), "=l"(r[4]), "=l"(r[5]), "=l"(r[6]), "=l"(r[7]), "=l"(r[8]), "=l"(r[9]), "=l"(r[10]), "=l"(r[11]), "=l"(r[12]), "=l"(r[13]), "=l"(r[14]), "=l"(r[15]), "=l"(r[16]), "=l"(r[17]), "=l"(r[18]), "=l"(r[19]), "=l"(r[20]), "=l"(r[21]), "=l"(r[22]), "=l"(r[23]), "=l"(r[24]), "=l"(r[25]), "=l"(r[26]), "=l"(r[27]), "=l"(r[28]), "=l"(r[29]), "=l"(r[30]), "=l"(r[31]) \
+      : "r"(taddr), "r"((taddr) + 32) \
       : "memory")
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -175,40 +210,111 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-
-// ---------------------------------------------------------------- kernel
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Barrier among the 256 softmax threads only (hardware barrier 1; barrier 0 is __syncthreads).
-__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Packed fp32 pairs (one 64-bit register pair; element 0 in the low half).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  return (uint64_t(__float_as_uint(hi)) << 32) | __float_as_uint(lo);
+}
+__device__ __forceinline__ float lo2(uint64_t v) { return __uint_as_float(uint32_t(v)); }
+__device__ __forceinline__ float hi2(uint64_t v) { return __uint_as_float(uint32_t(v >> 32)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Barrier between the two softmax warps that share a TMEM lane quadrant (hardware barrier
+// 1 + quadrant, 64 threads; barrier 0 is __syncthreads).  It also ANDs a predicate, so that both
+// take the same decision to go on or to give up.
+__device__ __forceinline__ bool pair_sync_and(int quadrant, bool ok) {
+  uint32_t res;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+      "bar.red.and.pred p, %1, 64, q;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(res) : "r"(quadrant + 1), "r"(uint32_t(ok)) : "memory");
+  return res != 0;
+}
 
+// Geometry of the key stream of one CTA, shared by the two producer warps.
+struct KeyStream {
+  const int32_t* sel;
+  const int32_t* pt;
+  int g_init, g_sel, g_past, gpb, n_cand, n_init, block, max_pages, n_phys_pages, page_base, page_oob;
+  int64_t local_start;
+};
+// Physical page (row of the 4-D tensor map) of 16-token granule gi of the past key stream;
+// page_oob (outside the tensor: TMA fills zeros) for padding granules and rejected indices.
+__device__ __forceinline__ int granule_page(const KeyStream& ks, int gi, int32_t* status, bool report) {
+  if (gi >= ks.g_past) return ks.page_oob;
+  int64_t lp;
+  if (gi < ks.g_init) {
+    lp = gi;
+  } else if (gi < ks.g_init + ks.g_sel) {
+    const int r = gi - ks.g_init;
+    const int blk = ks.sel[r / ks.gpb];
+    if (blk < 0 || blk >= ks.n_cand) {
+      if (report) set_status(status, ACTQKV_DEV_BAD_SELECTION);
+      return ks.page_oob;
+    }
+    lp = (int64_t(ks.n_init) + int64_t(blk) * ks.block) / 16 + r % ks.gpb;
+  } else {
+    lp = ks.local_start / 16 + (gi - ks.g_init - ks.g_sel);
+  }
+  const int phys = lp < ks.max_pages ? ks.pt[lp] : -1;
+  if (phys < 0 || phys >= ks.n_phys_pages) {
+    if (report) set_status(status, ACTQKV_DEV_BAD_PAGE);
+    return ks.page_oob;
+  }
+  return ks.page_base + phys;
+}
+
+// ---------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kw,
                     const __grid_constant__ CUtensorMap tm_vw, const __grid_constant__ CUtensorMap tm_kp,
                     const __grid_constant__ CUtensorMap tm_vp, TcParams p) {
   extern __shared__ unsigned char smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const bool smem_short = base - raw + kSmemNeeded > kSmemBytes;   // never with a 1 KiB-aligned window
   const uint32_t q_smem = base;
-  const uint32_t stage0 = base + kTileBytes;
-  const uint32_t bars = base + kSmemData;
+  const uint32_t k_ring = base + kTileBytes;
+  const uint32_t v_ring = k_ring + kRing * kTileBytes;
+  const uint32_t bars = base + kSmemTiles;
   // barrier slots (8 bytes each)
   const uint32_t bar_q = bars;
   auto bar_kfull = [&](int s) { return bars + 8u * (1 + s); };
-  auto bar_vfull = [&](int s) { return bars + 8u * (1 + kStages + s); };
-  auto bar_empty = [&](int s) { return bars + 8u * (1 + 2 * kStages + s); };
-  auto bar_sfull = [&](int b) { return bars + 8u * (1 + 3 * kStages + b); };
-  auto bar_pfull = [&](int b) { return bars + 8u * (3 + 3 * kStages + b); };
-  const uint32_t bar_done = bars + 8u * (5 + 3 * kStages);
-  unsigned char* base_generic = smem_raw + (base - smem_u32(smem_raw));
-  unsigned char* bars_generic = base_generic + kSmemData;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * (6 + 3 * kStages));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * (6 + 3 * kStages) + 8);
-  // after the last MMA has completed the Q tile is dead: its first 2 KiB carry the two
-  // warpgroups' (max, sum) pairs to the merge
-  float2* merge_ml = reinterpret_cast<float2*>(base_generic);
+  auto bar_kempty = [&](int s) { return bars + 8u * (1 + kRing + s); };
+  auto bar_vfull = [&](int s) { return bars + 8u * (1 + 2 * kRing + s); };
+  auto bar_vempty = [&](int s) { return bars + 8u * (1 + 3 * kRing + s); };
+  auto bar_sfull = [&](int b) { return bars + 8u * (1 + 4 * kRing + b); };
+  auto bar_pfull = [&](int b) { return bars + 8u * (1 + 4 * kRing + kSBuf + b); };
+  auto bar_pvdone = [&](int i) { return bars + 8u * (1 + 4 * kRing + 2 * kSBuf + i); };
+  const uint32_t bar_done = bars + 8u * (kNumBars - 1);
+  unsigned char* base_generic = smem_raw + (base - raw);
+  unsigned char* bars_generic = base_generic + kSmemTiles;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * kNumBars + 8);
+  float* xchg = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [2][2][128]
 
   const int mt = blockIdx.x, h = blockIdx.y, unit = blockIdx.z;
   const int g = h / p.group, seq = unit / p.n_layers, layer_local = unit - seq * p.n_layers;
@@ -223,22 +329,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     bad = true;
     c = max(0, min(c, min(p.cap_blocks, geo.n_cand)));
   }
-  const int gpb = p.block / 16;                          // page granules per block
-  const int g_init = geo.init_len / 16;
-  const int g_sel = c * gpb;
+  KeyStream ks;
+  ks.sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
+  ks.pt = p.a.page_table + size_t(seq) * p.max_pages;
+  ks.gpb = p.block / 16;                                 // page granules per block
+  ks.g_init = geo.init_len / 16;
+  ks.g_sel = c * ks.gpb;
   const int64_t local_len = geo.p0 - geo.local_start;
-  const int g_past = g_init + g_sel + int(local_len / 16);
-  const bool misaligned = (local_len % 16) != 0;
-  const int n_past = g_past * 16;
+  ks.g_past = ks.g_init + ks.g_sel + int(local_len / 16);
+  ks.n_cand = geo.n_cand; ks.n_init = p.n_init; ks.block = p.block; ks.max_pages = p.max_pages;
+  ks.n_phys_pages = p.n_phys_pages; ks.page_base = layer_local * p.n_phys_pages;
+  ks.page_oob = p.n_layers * p.n_phys_pages;             // beyond the tensor: zero fill
+  ks.local_start = geo.local_start;
+  const bool misaligned = (local_len % 16) != 0 || smem_short;
+  const int n_past = ks.g_past * 16;
   const int past_tiles = (n_past + kBN - 1) / kBN;
   const int n_tiles = past_tiles + mt + 1;
 
   if (tid == 0) {
-    if (bad) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
-    if (misaligned) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
+    if (bad || misaligned) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
     mbar_init(bar_q, 1);
-    for (int s = 0; s < kStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_vfull(s), 1); mbar_init(bar_empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 128); }
+    for (int s = 0; s < kRing; ++s) {
+      mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
+      mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
+    }
+    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 256); }
+    for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
     mbar_init(bar_done, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -257,177 +373,168 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     return;
   }
 
-  if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    if (warp == 0) {
-      // =========================== TMA producer ===========================
-      const int32_t* sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
-      const int32_t* pt = p.a.page_table + size_t(seq) * p.max_pages;
-      const int page_oob = p.n_layers * p.n_phys_pages;              // beyond the tensor: zero fill
-      if (lane == 0) {
-        mbar_expect_tx(bar_q, kTileBytes);
-        tma_load_3d(q_smem, &tm_q, bar_q, 0, h, unit * nt + mt * kBM);
-        tma_load_3d(q_smem + kSubTileBytes, &tm_q, bar_q, 64, h, unit * nt + mt * kBM);
-      }
-      bool ok = true;
-      int issued = 0;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j % kStages, it = j / kStages;
-        if (it > 0) ok = mbar_wait(bar_empty(s), (it - 1) & 1, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        const uint32_t sbase = stage0 + s * kStageBytes;
-        if (lane == 0) {
-          mbar_expect_tx(bar_kfull(s), kTileBytes);
-          mbar_expect_tx(bar_vfull(s), kTileBytes);
-        }
-        __syncwarp();
-        if (j < past_tiles) {
-          const int is_v = lane >> 4, half = (lane >> 3) & 1, slot = lane & 7;
-          const int gi = j * 8 + slot;
-          int page = page_oob;
-          if (gi < g_past) {
-            int64_t lp;
-            if (gi < g_init) {
-              lp = gi;
-            } else if (gi < g_init + g_sel) {
-              const int r = gi - g_init;
-              const int blk = sel[r / gpb];
-              lp = (blk >= 0 && blk < geo.n_cand) ? (int64_t(p.n_init) + int64_t(blk) * p.block) / 16 + r % gpb : -1;
-              if (lp < 0 && half == 0 && is_v == 0) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
-            } else {
-              lp = geo.local_start / 16 + (gi - g_init - g_sel);
-            }
-            if (lp >= 0) {
-              const int phys = lp < p.max_pages ? pt[lp] : -1;
-              if (phys < 0 || phys >= p.n_phys_pages) {
-                if (half == 0 && is_v == 0) set_status(p.a.status, ACTQKV_DEV_BAD_PAGE);
-              } else {
-                page = layer_local * p.n_phys_pages + phys;
-              }
-            }
-          }
-          const uint32_t dst = sbase + is_v * kTileBytes + half * kSubTileBytes + slot * 2048u;
-          tma_load_4d(dst, is_v ? &tm_vp : &tm_kp, is_v ? bar_vfull(s) : bar_kfull(s), half * 64, 0, g, page);
-        } else if (lane < 4) {
-          const int is_v = lane >> 1, half = lane & 1;
-          const int kt = j - past_tiles;
-          const uint32_t dst = sbase + is_v * kTileBytes + half * kSubTileBytes;
-          tma_load_3d(dst, is_v ? &tm_vw : &tm_kw, is_v ? bar_vfull(s) : bar_kfull(s), half * 64, g,
-                      unit * nt + kt * kBN);
-        }
-        issued = j + 1;
-      }
-      // drain: every issued copy must have landed before the CTA may exit on the abort path
-      if (!ok) {
-        for (int j = max(0, issued - kStages); j < issued; ++j) {
-          const int s = j % kStages, par = (j / kStages) & 1;
-          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_kfull(s), par); ++i) {}
-          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_vfull(s), par); ++i) {}
-        }
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
-      }
-    } else if (warp == 1) {
-      // =========================== MMA issuer ===========================
-      // Issue order QK(0), QK(1), PV(0), QK(2), PV(1), ...: the tensor pipe executes in issue
-      // order, so QK(j+2) cannot overwrite S/P buffer j&1 before PV(j) has read P(j), and a
-      // completed QK(j) implies a completed PV(j-2).
-      if (lane == 0) {
-        constexpr uint32_t idesc_qk = make_idesc(false);
-        constexpr uint32_t idesc_pv = make_idesc(true);
-        bool ok = mbar_wait(bar_q, 0, abort_flag);
-        auto issue_pv = [&](int i) {
-          const int s = i % kStages, b = i & 1;
-          ok = ok && mbar_wait(bar_vfull(s), (i / kStages) & 1, abort_flag);
-          ok = ok && mbar_wait(bar_pfull(b), (i >> 1) & 1, abort_flag);
-          if (!ok) return;
-          tc_fence_after();
-          const uint32_t vbase = stage0 + s * kStageBytes + kTileBytes;
-          const uint32_t p_tmem = tmem + b * 128;
-          const uint32_t o_tmem = tmem + 256 + b * 128;
-#pragma unroll
-          for (int k = 0; k < kBN / 16; ++k) {
-            // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
-            // term, then the 8 columns of the lo term of the same keys against the same V rows.
-            const uint64_t bdesc = make_desc(vbase + k * 2048u, kSubTileBytes, 1024u);
-            const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
-            mma_ts(o_tmem, pa, bdesc, idesc_pv, (i >= 2 || k > 0) ? 1u : 0u);
-            mma_ts(o_tmem, pa + 16, bdesc, idesc_pv, 1u);
-          }
-          tc_commit(bar_empty(s));
-        };
-        for (int j = 0; j < n_tiles && ok; ++j) {
-          const int s = j % kStages;
-          ok = mbar_wait(bar_kfull(s), (j / kStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t kbase = stage0 + s * kStageBytes;
-#pragma unroll
-          for (int k = 0; k < kD / 16; ++k) {
-            const uint32_t off = (k >> 2) * kSubTileBytes + (k & 3) * 32u;
-            const uint64_t adesc = make_desc(q_smem + off, 16u, 1024u);
-            const uint64_t bdesc = make_desc(kbase + off, 16u, 1024u);
-            mma_ss(tmem + (j & 1) * 128, adesc, bdesc, idesc_qk, k > 0 ? 1u : 0u);
-          }
-          tc_commit(bar_sfull(j & 1));
-          if (j >= 1) issue_pv(j - 1);
-        }
-        if (ok) issue_pv(n_tiles - 1);
-        if (ok) tc_commit(bar_done);
-      }
-      __syncwarp();
+  if (warp == 0 || warp == 2) {
+    // =========================== TMA producers: warp 0 -> K (and Q), warp 2 -> V ===========================
+    const bool is_v = warp == 2;
+    const uint32_t ring = is_v ? v_ring : k_ring;
+    const CUtensorMap* tm_pages = is_v ? &tm_vp : &tm_kp;
+    const CUtensorMap* tm_win = is_v ? &tm_vw : &tm_kw;
+    if (!is_v && lane == 0) {
+      mbar_expect_tx(bar_q, kTileBytes);
+      tma_load_3d(q_smem, &tm_q, bar_q, 0, h, unit * nt + mt * kBM);
+      tma_load_3d(q_smem + kSubTileBytes, &tm_q, bar_q, 64, h, unit * nt + mt * kBM);
     }
-  } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int half = (lane >> 3) & 1, slot = lane & 7;     // lanes 0-15: one box each
+    // Page lookups (sel_idx -> page_table, two dependent loads) are taken 32 granules = 4 tiles at
+    // a time, one granule per lane, one chunk ahead of the tiles being issued, so their latency
+    // is off the per-tile path; the issuing lane fetches its page with a shuffle.
+    auto resolve = [&](int chunk) {
+      const int gi = chunk * 32 + lane;
+      return gi < past_tiles * 8 ? granule_page(ks, gi, p.a.status, !is_v) : ks.page_oob;
+    };
+    int page_cur = 0, page_next = resolve(0);
+    bool ok = true;
+    int issued = 0;
+    for (int j = 0; j < n_tiles && ok; ++j) {
+      const int s = j % kRing, it = j / kRing;
+      if ((j & 3) == 0) {
+        page_cur = page_next;
+        page_next = resolve((j >> 2) + 1);
+      }
+      const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + slot);
+      if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const uint32_t full = is_v ? bar_vfull(s) : bar_kfull(s);
+      const uint32_t sbase = ring + s * kTileBytes;
+      if (lane == 0) mbar_expect_tx(full, kTileBytes);
+      __syncwarp();
+      if (j < past_tiles) {
+        if (lane < 16) tma_load_4d(sbase + half * kSubTileBytes + slot * 2048u, tm_pages, full, half * 64, 0, g, page);
+      } else if (lane < 2) {
+        tma_load_3d(sbase + lane * kSubTileBytes, tm_win, full, lane * 64, g, unit * nt + (j - past_tiles) * kBN);
+      }
+      issued = j + 1;
+    }
+    // drain: every issued copy must have landed before the CTA may exit on the abort path
+    if (!ok) {
+      for (int j = max(0, issued - kRing); j < issued; ++j) {
+        const uint32_t full = is_v ? bar_vfull(j % kRing) : bar_kfull(j % kRing);
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(full, (j / kRing) & 1); ++i) {}
+      }
+      if (!is_v) for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
+    }
+  } else if (warp == 1) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc(false);
+      constexpr uint32_t idesc_pv = make_idesc(true);
+      const uint32_t tmem_o = tmem + kSBuf * 128;
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      auto issue_qk = [&](int j) {
+        const int s = j % kRing;
+        ok = ok && mbar_wait(bar_kfull(s), (j / kRing) & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t kbase = k_ring + s * kTileBytes;
+        const uint32_t s_tmem = tmem + (j % kSBuf) * 128;
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k) {
+          const uint32_t off = (k >> 2) * kSubTileBytes + (k & 3) * 32u;
+          mma_ss(s_tmem, make_desc(q_smem + off, 16u, 1024u), make_desc(kbase + off, 16u, 1024u), idesc_qk,
+                 k > 0 ? 1u : 0u);
+        }
+        tc_commit(bar_kempty(s));
+        tc_commit(bar_sfull(j % kSBuf));
+      };
+      auto issue_pv = [&](int i) {
+        const int s = i % kRing, b = i % kSBuf;
+        ok = ok && mbar_wait(bar_vfull(s), (i / kRing) & 1, abort_flag);
+        ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t vbase = v_ring + s * kTileBytes;
+        const uint32_t p_tmem = tmem + b * 128;
+#pragma unroll
+        for (int k = 0; k < kBN / 16; ++k) {
+          // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
+          // term, then the 8 columns of the lo term of the same keys against the same V rows.
+          const uint64_t bdesc = make_desc(vbase + k * 2048u, kSubTileBytes, 1024u);
+          const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
+          mma_ts(tmem_o, pa, bdesc, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
+          mma_ts(tmem_o, pa + 16, bdesc, idesc_pv, 1u);
+        }
+        tc_commit(bar_vempty(s));
+        tc_commit(bar_pvdone(i % kPvRing));
+      };
+      issue_qk(0);
+      if (n_tiles > 1) issue_qk(1);
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        if (i + 2 < n_tiles) issue_qk(i + 2);
+        issue_pv(i);
+      }
+      if (ok) tc_commit(bar_done);
+    }
+    __syncwarp();
+  } else if (warp >= 4) {
     // =========================== softmax / epilogue ===========================
-    const int b = (warp >> 2) - 1;                        // 0: even tiles, 1: odd tiles
+    const int b = (warp >> 2) - 1;                        // column half of every tile
     const int q4 = warp & 3;                              // TMEM lane quadrant of this warp
     const int row = q4 * 32 + lane;                       // query row inside the tile
     const uint32_t lane_addr = uint32_t(q4 * 32) << 16;
-    const uint32_t s_addr = tmem + lane_addr + b * 128;
-    const uint32_t o_addr = tmem + lane_addr + 256 + b * 128;
+    const uint32_t o_addr = tmem + lane_addr + kSBuf * 128 + b * 64;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = b, kk = 0; j < n_tiles; j += 2, ++kk) {
-      ok = ok && mbar_wait(bar_sfull(b), kk & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int sb = j % kSBuf;
+      ok = ok && mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
       tc_fence_after();
-      uint32_t sr[128];
-      TMEM_LD128_WAIT(s_addr, sr);
+      const uint32_t s_addr = tmem + lane_addr + sb * 128 + b * 64;
+      uint64_t sv[32];
+      TMEM_LD64P_WAIT(s_addr, sv);
       // key-validity limit: ragged last past tile, or the causal diagonal of the last tile
       int limit = kBN;
       if (j < past_tiles) limit = min(kBN, n_past - j * kBN);
       else if (j == n_tiles - 1) limit = row + 1;
+      limit -= b * 64;                                    // in this thread's column numbering
       const bool masked = (j == n_tiles - 1) || (j == past_tiles - 1 && (n_past % kBN) != 0);   // CTA-uniform
-      float mx = -INFINITY;
+      float mx = -INFINITY, mx2 = -INFINITY;
       if (masked) {
 #pragma unroll
-        for (int i = 0; i < 128; ++i) {
-          const float x = i < limit ? __uint_as_float(sr[i]) : -INFINITY;
-          sr[i] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
+        for (int i = 0; i < 32; ++i) {
+          const float x0 = 2 * i < limit ? lo2(sv[i]) : -INFINITY;
+          const float x1 = 2 * i + 1 < limit ? hi2(sv[i]) : -INFINITY;
+          sv[i] = pack2(x0, x1);
+          mx = max3(mx, x0, x1);
         }
       } else {
-        float mx2 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 128; i += 2) {
-          mx = fmaxf(mx, __uint_as_float(sr[i]));
-          mx2 = fmaxf(mx2, __uint_as_float(sr[i + 1]));
+        for (int i = 0; i < 32; i += 2) {
+          mx = max3(mx, lo2(sv[i]), hi2(sv[i]));
+          mx2 = max3(mx2, lo2(sv[i + 1]), hi2(sv[i + 1]));
         }
         mx = fmaxf(mx, mx2);
       }
+      // the row's maximum over both column halves
+      float* xrow = xchg + (j & 1) * 256 + row;
+      xrow[b * 128] = mx;
+      ok = pair_sync_and(q4, ok);
+      if (!ok) break;                                     // both threads of a row leave together
+      mx = fmaxf(mx, xrow[(1 - b) * 128]);
       const float m_new = fmaxf(m_used, mx * p.scale_log2);
       const bool grow = m_new - m_used > kRescaleThreshold;     // also true for the first tile
-      if (kk == 0) {
+      if (j == 0) {
         m_used = m_new;
       } else if (__any_sync(0xffffffffu, grow)) {
-        // S(j) complete implies PV(j-2) complete: this warpgroup's O is quiescent until it
-        // publishes P(j)
+        // O must be quiescent: P V of every earlier tile complete (tile j's is not issued before
+        // this thread publishes P(j)).  One barrier per tile in a ring of 4, so the parity of the
+        // awaited phase cannot be confused with a later one.
+        ok = mbar_wait(bar_pvdone((j - 1) % kPvRing), ((j - 1) / kPvRing) & 1, abort_flag);
+        tc_fence_after();
         const float f = grow ? ex2(m_used - m_new) : 1.f;
         if (grow) { m_used = m_new; l *= f; }
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cc = 0; cc < 2; ++cc) {
           uint32_t orr[32];
           TMEM_LD32_WAIT(o_addr + cc * 32, orr);
 #pragma unroll
@@ -437,78 +544,70 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
       // P = exp2(x - m) split into two bf16 terms (hi + lo): with outlier value channels a
       // single bf16 P (8 significant bits) would cost up to |v| * 2^-9 of absolute error.
-      const float neg_m = -m_used;
-      float sum0 = 0.f, sum1 = 0.f;
+      const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm2 = pack2(-m_used, -m_used);
+      uint64_t sum_a = 0, sum_b = 0;                      // two (+0, +0) pairs
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
+      for (int cc = 0; cc < 2; ++cc) {
         uint32_t pk[32];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const float e0 = ex2(fmaf(__uint_as_float(sr[32 * cc + 2 * i]), p.scale_log2, neg_m));
-          const float e1 = ex2(fmaf(__uint_as_float(sr[32 * cc + 2 * i + 1]), p.scale_log2, neg_m));
-          sum0 += e0;
-          sum1 += e1;
+          const uint64_t x = fma2(sv[16 * cc + i], scale2, negm2);
+          const float e0 = ex2(lo2(x)), e1 = ex2(hi2(x));
+          const uint64_t e = pack2(e0, e1);
+          if (i & 1) sum_b = add2(sum_b, e); else sum_a = add2(sum_a, e);
           const uint32_t hi = pack_bf16(e0, e1);
           pk[i] = hi;
-          pk[16 + i] = pack_bf16(e0 - __uint_as_float(hi << 16), e1 - __uint_as_float(hi & 0xFFFF0000u));
+          const uint64_t lo = sub2(e, (uint64_t(hi & 0xFFFF0000u) << 32) | (hi << 16));
+          pk[16 + i] = pack_bf16(lo2(lo), hi2(lo));
         }
         TMEM_ST32(s_addr + cc * 32, pk);
       }
-      l += sum0 + sum1;
+      sum_a = add2(sum_a, sum_b);
+      l += lo2(sum_a) + hi2(sum_a);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_pfull(b));
+      mbar_arrive(bar_pfull(sb));
     }
-    // ---- merge of the two warpgroups' partial results and epilogue
+    // ---- epilogue: the row sum over both column halves, then this thread's 64 channels of O / l
     ok = ok && mbar_wait(bar_done, 0, abort_flag);
-    if (ok) merge_ml[b * 128 + row] = make_float2(m_used, l);
-    softmax_sync();
-    if (*abort_flag == 0) {
+    float* xrow = xchg + (n_tiles & 1) * 256 + row;
+    xrow[b * 128] = l;
+    ok = pair_sync_and(q4, ok);
+    if (ok) {
       tc_fence_after();
-      const float2 a0 = merge_ml[row], a1 = merge_ml[128 + row];
-      const float m = fmaxf(a0.x, a1.x);
-      float f0 = a0.y > 0.f ? ex2(a0.x - m) : 0.f;
-      float f1 = a1.y > 0.f ? ex2(a1.x - m) : 0.f;
-      const float lsum = a0.y * f0 + a1.y * f1;
+      const float lsum = l + xrow[(1 - b) * 128];
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-      f0 *= inv;
-      f1 *= inv;
-      const bool use1 = f1 != 0.f;                          // O1 was never written when the CTA has one tile
       const size_t tok = size_t(unit) * nt + size_t(mt) * kBM + row;
-      const uint32_t o0 = tmem + lane_addr + 256, o1 = tmem + lane_addr + 384;
 #pragma unroll
       for (int cc = 0; cc < 2; ++cc) {
-        const int col = b * 64 + cc * 32;                   // this warpgroup's half of the channels
-        uint32_t r0[32], r1[32];
-        TMEM_LD32_WAIT(o0 + col, r0);
-        TMEM_LD32_WAIT(o1 + col, r1);
-        float o[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float x1 = use1 ? __uint_as_float(r1[i]) * f1 : 0.f;
-          o[i] = fmaf(__uint_as_float(r0[i]), f0, x1);
-        }
+        const int col = b * 64 + cc * 32;
+        uint32_t orr[32];
+        TMEM_LD32_WAIT(o_addr + cc * 32, orr);
         if (p.out_bf16) {
           __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             uint4 v;
-            v.x = pack_bf16(o[8 * i + 0], o[8 * i + 1]);
-            v.y = pack_bf16(o[8 * i + 2], o[8 * i + 3]);
-            v.z = pack_bf16(o[8 * i + 4], o[8 * i + 5]);
-            v.w = pack_bf16(o[8 * i + 6], o[8 * i + 7]);
+            v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
             *reinterpret_cast<uint4*>(ob + 8 * i) = v;
           }
         } else {
           float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            *reinterpret_cast<float4*>(of + 4 * i) = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          for (int i = 0; i < 8; ++i) {
+            float4 v;
+            v.x = __uint_as_float(orr[4 * i + 0]) * inv; v.y = __uint_as_float(orr[4 * i + 1]) * inv;
+            v.z = __uint_as_float(orr[4 * i + 2]) * inv; v.w = __uint_as_float(orr[4 * i + 3]) * inv;
+            *reinterpret_cast<float4*>(of + 4 * i) = v;
+          }
         }
       }
       if (p.a.lse && b == 0)
         p.a.lse[(size_t(unit) * p.n_q_heads + h) * nt + size_t(mt) * kBM + row] =
-            (m + log2f(lsum)) * 0.6931471805599453f;
+            (m_used + log2f(lsum)) * 0.6931471805599453f;
     }
   }
 
