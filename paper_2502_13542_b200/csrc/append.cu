@@ -3,9 +3,10 @@
 // One launch, two roles selected by blockIdx.x:
 //   copy CTAs   scatter the step's K / V rows into their pages (16-byte vectors);
 //   repr CTAs   one per (completed block, KV head): each of the r representatives is the
-//               mean of B/r consecutive keys, accumulated in fp64 (exact for bf16 inputs, so
-//               the rounded table is bit-reproducible), rounded to the cache dtype; the
-//               inverse norm is taken from the rounded values.  Keys older than the step are
+//               mean of B/r consecutive keys, read as 16-byte vectors by all threads at once
+//               and accumulated in fp64 (exact for bf16 inputs, so the rounded table is
+//               bit-reproducible), rounded to the cache dtype; the inverse norm is taken from
+//               the rounded values in a fixed order.  Keys older than the step are
 //               read from the pages, the step's own keys from k_win, so the two roles do not
 //               depend on each other.
 #include "common.cuh"
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
     return;
   }
 
-  // ---- repr role
+  // ---- repr role: one CTA per (completed block, KV head)
   const int rid = blockIdx.x - p.copy_ctas;
   const int g = rid % p.n_kv_heads, nb = rid / p.n_kv_heads;
   const int64_t p1 = p0 + p.n_tokens;
@@ -77,50 +78,63 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
     if (tid == 0) set_status(p.status, ACTQKV_DEV_TABLE_FULL);
     return;
   }
-  __shared__ float sq_s[kThreads];
+  // Thread t owns the 16-byte channel vector cv of rows rsub, rsub + rpp, ... of each chunk; the
+  // rpp partial sums of a channel are then added in a fixed order.  fp64 throughout: exact for
+  // bf16 keys, so the rounded table does not depend on the order.
+  extern __shared__ __align__(16) unsigned char append_smem[];
+  double* red = reinterpret_cast<double*>(append_smem);            // [rpp][D]
+  float* sq_s = reinterpret_cast<float*>(red + size_t(kThreads / vpr) * D);   // [D]
+  const int rpp = kThreads / vpr;                                   // rows per pass
+  const int cv = tid % vpr, rsub = tid / vpr;
   const int seg = p.block / p.n_repr;
   const size_t row0 = ((size_t(unit) * p.n_kv_heads + g) * p.n_cap + size_t(b)) * p.n_repr;
   T* tab = static_cast<T*>(p.repr_k) + row0 * D;
-  // threads cover (representative i, channel c); loop when r * D > kThreads
-  for (int base = 0; base < p.n_repr * D; base += kThreads) {
-    const int e = base + tid;
-    const int i = e / D, cch = e - i * D;
-    float stored = 0.f;
-    if (e < p.n_repr * D) {
-      const int64_t t0 = int64_t(p.n_init) + b * p.block + int64_t(i) * seg;
-      const int64_t tlo = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? t0 : t0 + seg / 2;
-      const int64_t thi = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? t0 + seg : tlo + 1;
-      double acc = 0.0;
-      for (int64_t tok = tlo; tok < thi; ++tok) {
-        float v = 0.f;
-        if (tok >= p0) {
-          v = to_f32(kw[(size_t(tok - p0) * p.n_kv_heads + g) * D + cch]);
+  const int64_t blk0 = int64_t(p.n_init) + b * p.block;
+  for (int i = 0; i < p.n_repr; ++i) {
+    const int lo = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? i * seg : i * seg + seg / 2;
+    const int hi = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? (i + 1) * seg : lo + 1;
+    double acc[VN];
+#pragma unroll
+    for (int e = 0; e < VN; ++e) acc[e] = 0.0;
+    for (int r = lo + rsub; r < hi; r += rpp) {
+      const int64_t tok = blk0 + r;
+      const T* src = nullptr;
+      if (tok >= p0) {
+        src = kw + (size_t(tok - p0) * p.n_kv_heads + g) * D + cv * VN;
+      } else {
+        const int64_t lp = tok / p.page_tokens;
+        const int phys = lp < p.max_pages ? pt[lp] : -1;
+        if (phys < 0 || phys >= p.n_phys_pages) {
+          if (cv == 0) set_status(p.status, ACTQKV_DEV_BAD_PAGE);
         } else {
-          const int64_t lp = tok / p.page_tokens;
-          const int phys = lp < p.max_pages ? pt[lp] : -1;
-          if (phys < 0 || phys >= p.n_phys_pages) {
-            if (cch == 0) set_status(p.status, ACTQKV_DEV_BAD_PAGE);
-          } else {
-            v = to_f32(kp[(size_t(phys) * p.n_kv_heads + g) * p.page_tokens * D +
-                          size_t(tok % p.page_tokens) * D + cch]);
-          }
+          src = kp + (size_t(phys) * p.n_kv_heads + g) * p.page_tokens * D + size_t(tok % p.page_tokens) * D + cv * VN;
         }
-        acc += double(v);
       }
-      const double mean = acc / double(thi - tlo);
+      if (src) {
+        float kf[VN];
+        Vec16<T>::load_nc(src, kf);
+#pragma unroll
+        for (int e = 0; e < VN; ++e) acc[e] += double(kf[e]);
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < VN; ++e) red[size_t(rsub) * D + cv * VN + e] = acc[e];
+    __syncthreads();
+    if (tid < D) {
+      double t = 0.0;
+      for (int q = 0; q < rpp; ++q) t += red[size_t(q) * D + tid];
+      const double mean = t / double(hi - lo);
       const T rounded = from_f32<T>(float(mean));   // fp64 -> fp32 -> dtype, both nearest-even
-      tab[size_t(i) * D + cch] = rounded;
-      stored = to_f32(rounded);
-    }
-    // inverse norms of the representatives covered by this pass (D threads each)
-    sq_s[tid] = stored * stored;
-    __syncthreads();
-    if (tid < kThreads / D && base / D + tid < p.n_repr) {
-      float s = 0.f;
-      for (int cc = 0; cc < D; ++cc) s += sq_s[tid * D + cc];
-      p.repr_inv_norm[row0 + base / D + tid] = s > 0.f ? rsqrtf(s) : 0.f;
+      tab[size_t(i) * D + tid] = rounded;
+      const float stored = to_f32(rounded);
+      sq_s[tid] = stored * stored;
     }
     __syncthreads();
+    if (tid == 0) {
+      float t = 0.f;
+      for (int cc = 0; cc < D; ++cc) t += sq_s[cc];
+      p.repr_inv_norm[row0 + i] = t > 0.f ? rsqrtf(t) : 0.f;
+    }
   }
 }
 
@@ -154,7 +168,8 @@ extern "C" int actqkv_append_window(const actqkv_config* cfg, const actqkv_batch
   p.max_new_blocks = n_tokens / cfg->block + 2;
   dim3 grid(p.copy_ctas + p.max_new_blocks * cfg->n_kv_heads, b.units());
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (cfg->dtype == ACTQKV_BF16) append_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(p);
-  else append_kernel<float><<<grid, kThreads, 0, st>>>(p);
+  const size_t smem = sizeof(double) * size_t(kThreads / vpr) * cfg->head_dim + sizeof(float) * cfg->head_dim;
+  if (cfg->dtype == ACTQKV_BF16) append_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(p);
+  else append_kernel<float><<<grid, kThreads, smem, st>>>(p);
   return launch_status();
 }

@@ -1,12 +1,17 @@
 // Steps 1 and 2: Activation Bias (Eq. 7, statistics Eq. 8) and the activation-aware
 // probe-query (Eq. 9).
 //
-// One CTA per (unit, query head).  The head's [n_tokens x D] query tile is read from HBM
-// once into shared memory (rows of D elements, 16-byte loads); the window's per-channel
-// mean and sum of squared deviations are taken two-pass from shared memory and merged
-// into the running statistics, so Eq. 8 over all windows costs one HBM pass per window.
-// The G CTAs of one KV head form a thread-block cluster; rank 0 averages the G probes
-// through distributed shared memory in a fixed order (bitwise reproducible).
+// The [n_tokens x D] query tile of one (unit, query head) is split by rows over S CTAs, and the
+// S x G CTAs of one KV head form a thread-block cluster (S * G <= 8).  Every CTA brings its rows from HBM into shared memory with one
+// bulk asynchronous copy per row (all in flight at once) and makes three passes over them with
+// 16-byte shared-memory loads:
+//   1. per-channel sums of q and of (q - shift)^2, shift = the CTA's first row, which give
+//      the mean and the sum of squared deviations of its rows without a second pass; the row
+//      splits are merged pairwise (count, mean, M2) in a fixed order through distributed shared
+//      memory and then merged into the running statistics (Eq. 8 over all windows so far);
+//   2. phi and the per-token indicator ||phi_j||_1 (Eq. 7);
+//   3. sum_j a_j q_j, combined with sum_j a_j by the group leaders in a fixed order (Eq. 9).
+// Every reduction order is fixed, so results are bitwise reproducible.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -17,10 +22,13 @@ using namespace actqkv;
 namespace {
 
 constexpr int kThreads = 512;
+constexpr int kMaxCluster = 8;
+constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct BiasProbeParams {
   const void* q;
   int n_tokens, n_q_heads, n_kv_heads, head_dim, group;
+  int split, rows_per_cta;
   int64_t* stats_count;
   float* stats_mean;
   float* stats_m2;
@@ -35,186 +43,313 @@ struct BiasProbeParams {
   int32_t* status;
 };
 
-__device__ __forceinline__ float block_sum(float v, float* scratch) {
-  v = warp_sum(v);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  __syncthreads();
-  if (lane == 0) scratch[warp] = v;
-  __syncthreads();
-  float t = 0.f;
-  for (int i = 0; i < kThreads / 32; ++i) t += scratch[i];   // same order in every thread
-  return t;
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-template <typename T, bool kCluster>
+template <typename T, int D>
 __global__ void __launch_bounds__(kThreads) bias_probe_kernel(BiasProbeParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int D = p.head_dim, W = p.n_tokens;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  cg::cluster_group cluster = cg::this_cluster();
+  constexpr int VN = Vec16<T>::N;             // elements per 16-byte vector
+  constexpr int VPR = D / VN;                 // vectors per row
+  constexpr int RL = kThreads / VPR;          // row lanes: thread (cv, rsub) owns vector cv of rows rsub + k * RL
+  constexpr int NP = kThreads / D;            // second-level slices of the row lanes
+  constexpr int PER = RL / NP;
+  const int W = p.n_tokens, S = p.split, RP = p.rows_per_cta;
   T* tile = reinterpret_cast<T*>(smem_raw);
-  float* fbase = reinterpret_cast<float*>(smem_raw + ((size_t(W) * D * sizeof(T) + 15) & ~size_t(15)));
-  const int R = kThreads / D;                 // row groups for column passes
-  float* partial = fbase;                     // [R][D]
-  float* mean_s = partial + R * D;            // [D]
+  float* partial = reinterpret_cast<float*>(smem_raw + ((size_t(RP) * D * sizeof(T) + 127) & ~size_t(127)));   // [2][RL][D]
+  float* level2 = partial + 2 * RL * D;       // [2][NP][D]
+  // records read by other CTAs of the cluster (same offsets in every CTA)
+  float* st_mean = level2 + 2 * NP * D;       // [D] mean of this CTA's rows
+  float* st_m2 = st_mean + D;                 // [D] sum of squared deviations about it
+  float* u_s = st_m2 + D;                     // [D] sum_j a_j q_j over this CTA's rows
+  float* qsum_s = u_s + D;                    // [D] sum_j q_j over this CTA's rows
+  float* scal = qsum_s + D;                   // [0] = sum_j a_j, [1] = rows held
+  float* mean_s = scal + 4;                   // [D]
   float* ivar_s = mean_s + D;                 // [D]
-  float* probe_s = ivar_s + D;                // [D]
-  float* red_s = probe_s + D;                 // [32]
-  float* a_s = red_s + 32;                    // [W]
+  float* red_s = ivar_s + D;                  // [32]
+  float* a_s = red_s + 32;                    // [RP]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(a_s + ((RP + 3) & ~3));
 
-  const int h = blockIdx.x, unit = blockIdx.y;
+  const int sp = blockIdx.x, h = blockIdx.y, unit = blockIdx.z;
+  const int hy = h % p.group;                 // head inside its KV group
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const T* qbase = reinterpret_cast<const T*>(p.q) + (size_t(unit) * W * p.n_q_heads + h) * D;
+  const int r0 = min(W, sp * RP), nr = min(W, r0 + RP) - r0;      // this CTA's rows [r0, r0 + nr)
   const size_t row_stride = size_t(p.n_q_heads) * D;
-  constexpr int VN = Vec16<T>::N;
-  const int vec_per_row = D / VN;
+  const T* qbase = reinterpret_cast<const T*>(p.q) + (size_t(unit) * W + r0) * row_stride + size_t(h) * D;
+  const int cy = p.do_probe ? p.group : 1;    // cluster = (S, cy): rank of (split s, head-in-group y) = s + S * y
+  const size_t hd = (size_t(unit) * p.n_q_heads + h) * D;
+  const size_t uh = size_t(unit) * p.n_q_heads + h;
 
-  // ---- 1. tile -> shared memory, one HBM pass
-  for (int idx = tid; idx < W * vec_per_row; idx += kThreads) {
-    const int row = idx / vec_per_row, cv = idx - row * vec_per_row;
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(qbase + row * row_stride + cv * VN));
-    *reinterpret_cast<uint4*>(tile + size_t(row) * D + cv * VN) = v;
+  // ---- 0. rows -> shared memory: one bulk copy per row, all in flight together
+  constexpr uint32_t kRowBytes = D * sizeof(T);
+  const uint32_t bar_addr = smem_addr(bar);
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  if (tid == 0 && nr > 0)
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(uint32_t(nr) * kRowBytes) : "memory");
+  __syncthreads();
+  for (int r = tid; r < nr; r += kThreads)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(tile + size_t(r) * D)), "l"(qbase + size_t(r) * row_stride), "r"(kRowBytes), "r"(bar_addr)
+                 : "memory");
+  // running statistics of this head, fetched while the copies fly
+  const bool running = p.do_bias && p.stats_mode == ACTQKV_STATS_CUMULATIVE;
+  float run_mean = 0.f, run_m2 = 0.f;
+  int64_t run_count = 0;
+  if (running && tid < D) {
+    run_mean = p.stats_mean[hd + tid];
+    run_m2 = p.stats_m2[hd + tid];
+    run_count = p.stats_count[uh];
+  }
+  if (nr > 0) {
+    bool landed = false;
+    for (uint32_t i = 0; i < kSpinLimit && !landed; ++i) {
+      uint32_t ok;
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                   : "=r"(ok) : "r"(bar_addr) : "memory");
+      landed = ok != 0;
+    }
+    if (!landed && tid == 0) set_status(p.status, ACTQKV_DEV_TIMEOUT);     // goes on with whatever arrived
+  }
 
-  const int c = tid % D, rg = tid / D;
-  const size_t hd = (size_t(unit) * p.n_q_heads + h) * D;
+  const int cv = tid % VPR, rsub = tid / VPR;
+  const int n_pass = (nr + RL - 1) / RL;      // same trip count in every thread
+  auto load_row = [&](int r, float (&f)[VN]) { Vec16<T>::load(tile + size_t(r) * D + cv * VN, f); };
+  // dst_k[D] = sum over the row lanes of acc_k, k < NA, in a fixed two-level order
+  auto column_reduce2 = [&](const float (&a0)[VN], const float (&a1)[VN], float* dst0, float* dst1) {
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < VN; ++e) {
+      partial[rsub * D + cv * VN + e] = a0[e];
+      partial[RL * D + rsub * D + cv * VN + e] = a1[e];
+    }
+    __syncthreads();
+    {
+      const int ch = tid % D, part = tid / D;
+      float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < PER; ++q) {
+        t0 += partial[(part * PER + q) * D + ch];
+        t1 += partial[RL * D + (part * PER + q) * D + ch];
+      }
+      level2[part * D + ch] = t0;
+      level2[NP * D + part * D + ch] = t1;
+    }
+    __syncthreads();
+    if (tid < D) {
+      float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < NP; ++q) { t0 += level2[q * D + tid]; t1 += level2[NP * D + q * D + tid]; }
+      dst0[tid] = t0;
+      dst1[tid] = t1;
+    }
+    __syncthreads();
+  };
+
+  // ---- 1. shifted first and second moments of this CTA's rows
+  {
+    float shift[VN], s1[VN], s2[VN];
+#pragma unroll
+    for (int e = 0; e < VN; ++e) { s1[e] = 0.f; s2[e] = 0.f; shift[e] = 0.f; }
+    if (nr > 0) load_row(0, shift);
+    for (int r = rsub; r < nr; r += RL) {
+      float f[VN];
+      load_row(r, f);
+#pragma unroll
+      for (int e = 0; e < VN; ++e) { const float d = f[e] - shift[e]; s1[e] += f[e]; s2[e] = fmaf(d, d, s2[e]); }
+    }
+    column_reduce2(s1, s2, st_mean, st_m2);      // for now: sum q and sum (q - shift)^2
+    if (tid < D) {
+      const double n = double(nr), sh0 = nr > 0 ? double(to_f32(tile[tid])) : 0.0;
+      const double sq = double(st_mean[tid]), b2 = double(st_m2[tid]);
+      const double a = sq - n * sh0;             // sum (q - shift)
+      qsum_s[tid] = st_mean[tid];
+      st_mean[tid] = nr > 0 ? float(sq / n) : 0.f;
+      st_m2[tid] = nr > 0 ? float(fmax(b2 - a * a / n, 0.0)) : 0.f;
+    }
+    if (tid == 0) scal[1] = float(nr);
+  }
 
   if (p.do_bias) {
-    // ---- 2. window mean and M2 per channel (two passes over shared memory)
-    float s = 0.f;
-    for (int r = rg; r < W; r += R) s += to_f32(tile[size_t(r) * D + c]);
-    partial[rg * D + c] = s;
-    __syncthreads();
-    float wmean = 0.f;
+    cluster.sync();
+    // ---- 2. merge the row splits, then the running statistics (Eq. 8 over all windows so far)
     if (tid < D) {
-      for (int i = 0; i < R; ++i) wmean += partial[i * D + tid];
-      wmean /= float(W);
-      mean_s[tid] = wmean;
-    }
-    __syncthreads();
-    const float mc = mean_s[c];
-    s = 0.f;
-    for (int r = rg; r < W; r += R) {
-      const float d = to_f32(tile[size_t(r) * D + c]) - mc;
-      s = fmaf(d, d, s);
-    }
-    __syncthreads();
-    partial[rg * D + c] = s;
-    __syncthreads();
-    // ---- 3. merge into the running statistics (Eq. 8 over all windows so far)
-    if (tid < D) {
-      double m2w = 0.0;
-      for (int i = 0; i < R; ++i) m2w += double(partial[i * D + tid]);
-      double mean = double(mean_s[tid]), m2 = m2w, n = double(W);
-      if (p.stats_mode == ACTQKV_STATS_CUMULATIVE) {
-        const double na = double(p.stats_count[size_t(unit) * p.n_q_heads + h]);
-        const double mean_a = double(p.stats_mean[hd + tid]), m2_a = double(p.stats_m2[hd + tid]);
-        n = na + double(W);
-        const double delta = mean - mean_a;
-        mean = mean_a + delta * (double(W) / n);
-        m2 = m2_a + m2w + delta * delta * (na * double(W) / n);
-        p.stats_mean[hd + tid] = float(mean);
-        p.stats_m2[hd + tid] = float(m2);
+      float pn[kMaxCluster], pm[kMaxCluster], pm2[kMaxCluster];
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+        pn[s2] = 0.f; pm[s2] = 0.f; pm2[s2] = 0.f;
+        if (s2 < S) {
+          const unsigned rk = unsigned(s2 + S * (cy > 1 ? hy : 0));
+          pn[s2] = cluster.map_shared_rank(scal, rk)[1];
+          pm[s2] = cluster.map_shared_rank(st_mean, rk)[tid];
+          pm2[s2] = cluster.map_shared_rank(st_m2, rk)[tid];
+        }
+      }
+      double n = 0.0, mean = 0.0, m2 = 0.0;
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+        const double nb = double(pn[s2]);
+        if (nb == 0.0) continue;
+        const double nn = n + nb, delta = double(pm[s2]) - mean, w = nb / nn;
+        mean += delta * w;
+        m2 += double(pm2[s2]) + delta * delta * (n * w);
+        n = nn;
+      }
+      if (running) {
+        const double na = double(run_count), mean_a = double(run_mean), m2_a = double(run_m2);
+        const double nn = na + n, delta = mean - mean_a, w = n / nn;
+        mean = mean_a + delta * w;
+        m2 = m2_a + m2 + delta * delta * (na * w);
+        n = nn;
+        if (sp == 0) {                         // every CTA took the old values at kernel start
+          p.stats_mean[hd + tid] = float(mean);
+          p.stats_m2[hd + tid] = float(m2);
+          if (tid == 0) p.stats_count[uh] = run_count + W;
+        }
       }
       const double var = n > 1.0 ? m2 / (n - 1.0) : 0.0;
       mean_s[tid] = float(mean);
       ivar_s[tid] = float(1.0 / fmax(var, double(p.var_eps)));
     }
     __syncthreads();
-    if (tid == 0 && p.stats_mode == ACTQKV_STATS_CUMULATIVE)
-      p.stats_count[size_t(unit) * p.n_q_heads + h] += W;
-    // ---- 4. phi and its L1 norm per token: one warp per row
-    for (int r = warp; r < W; r += kThreads / 32) {
-      float acc = 0.f;
-      for (int cc = lane; cc < D; cc += 32) {
-        const float d = to_f32(tile[size_t(r) * D + cc]) - mean_s[cc];
-        const float ph = d * d * ivar_s[cc];
-        acc += ph;
-        if (p.phi_full) p.phi_full[(size_t(unit) * W + r) * row_stride + size_t(h) * D + cc] = ph;
-      }
-      acc = warp_sum(acc);
-      if (lane == 0) {
-        a_s[r] = acc;
-        if (p.phi_l1) p.phi_l1[(size_t(unit) * p.n_q_heads + h) * W + r] = acc;
+    // ---- 3. phi and its L1 norm per token: the VPR lanes of a row add up by shuffles
+    {
+      float mc[VN], iv[VN];
+#pragma unroll
+      for (int e = 0; e < VN; ++e) { mc[e] = mean_s[cv * VN + e]; iv[e] = ivar_s[cv * VN + e]; }
+      for (int k = 0; k < n_pass; ++k) {
+        const int r = rsub + k * RL;
+        float part = 0.f;
+        if (r < nr) {
+          float f[VN], ph[VN];
+          load_row(r, f);
+#pragma unroll
+          for (int e = 0; e < VN; ++e) { const float d = f[e] - mc[e]; ph[e] = d * d * iv[e]; part += ph[e]; }
+          if (p.phi_full) {
+            float* dst = p.phi_full + (size_t(unit) * W + r0 + r) * row_stride + size_t(h) * D + cv * VN;
+#pragma unroll
+            for (int e = 0; e < VN; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(ph[e], ph[e + 1], ph[e + 2], ph[e + 3]);
+          }
+        }
+#pragma unroll
+        for (int o = VPR >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if (r < nr && cv == 0) a_s[r] = part;
       }
     }
+    __syncthreads();
+    if (p.phi_l1)
+      for (int r = tid; r < nr; r += kThreads) p.phi_l1[uh * W + r0 + r] = a_s[r];
   } else {
-    for (int r = tid; r < W; r += kThreads) a_s[r] = p.phi_l1[(size_t(unit) * p.n_q_heads + h) * W + r];
+    for (int r = tid; r < nr; r += kThreads) a_s[r] = p.phi_l1[uh * W + r0 + r];
+    __syncthreads();
   }
-  __syncthreads();
-  if (!p.do_probe) return;
+  if (!p.do_probe) {
+    if (p.do_bias) cluster.sync();      // peers may still be reading this CTA's record in step 2
+    return;
+  }
 
-  // ---- 5. weights ||phi_j||_1 / ||Phi||_1
-  float part = 0.f;
-  for (int r = tid; r < W; r += kThreads) part += a_s[r];
-  const float total = block_sum(part, red_s);
-  const bool uniform = !(total > 0.f);
-  const float inv_total = uniform ? 0.f : 1.f / total;
-  const float wu = 1.f / float(W);
-  // ---- 6. probe = sum_j w_j q_j, column pass
-  float s = 0.f;
-  for (int r = rg; r < W; r += R) {
-    const float w = uniform ? wu : a_s[r] * inv_total;
-    s = fmaf(w, to_f32(tile[size_t(r) * D + c]), s);
-  }
-  __syncthreads();
-  partial[rg * D + c] = s;
-  __syncthreads();
-  if (tid < D) {
-    float pr = 0.f;
-    for (int i = 0; i < R; ++i) pr += partial[i * D + tid];
-    probe_s[tid] = pr;
-    p.probe_qh[hd + tid] = pr;
-  }
-  // ---- 7. KV-head probe: mean over the G query heads of the group, via DSMEM
-  if constexpr (kCluster) {
-    cg::cluster_group cluster = cg::this_cluster();
-    cluster.sync();
-    if (cluster.block_rank() == 0 && tid < D) {
-      float acc = 0.f;
-      for (int r = 0; r < p.group; ++r) acc += cluster.map_shared_rank(probe_s, r)[tid];
-      const int g = h / p.group;
-      p.probe_kv[(size_t(unit) * p.n_kv_heads + g) * D + tid] = acc / float(p.group);
+  // ---- 4. this CTA's share of ||Phi||_1 and of sum_j a_j q_j
+  {
+    float part = 0.f;
+    for (int r = tid; r < nr; r += kThreads) part += a_s[r];
+    part = warp_sum(part);
+    if (lane == 0) red_s[warp] = part;
+    float acc[VN], zero[VN];
+#pragma unroll
+    for (int e = 0; e < VN; ++e) { acc[e] = 0.f; zero[e] = 0.f; }
+    for (int r = rsub; r < nr; r += RL) {
+      float f[VN];
+      load_row(r, f);
+      const float w = a_s[r];
+#pragma unroll
+      for (int e = 0; e < VN; ++e) acc[e] = fmaf(w, f[e], acc[e]);
     }
-    cluster.sync();
+    column_reduce2(acc, zero, u_s, mean_s);      // mean_s is free by now: dummy destination
+    if (tid == 0) {
+      float t = 0.f;
+      for (int i = 0; i < kThreads / 32; ++i) t += red_s[i];
+      scal[0] = t;
+    }
   }
+  cluster.sync();
+  // ---- 5. Eq. 9 per query head, and the KV-head probe = mean over the G heads of the group.
+  // The group leader repeats the per-head arithmetic in the same order, so both agree bitwise.
+  if (sp == 0 && tid < D) {
+    float tot[kMaxCluster], uu[kMaxCluster], qq[kMaxCluster];
+    const int n_cta = S * cy;
+#pragma unroll
+    for (int rk = 0; rk < kMaxCluster; ++rk) {
+      tot[rk] = 0.f; uu[rk] = 0.f; qq[rk] = 0.f;
+      if (rk < n_cta && (hy == 0 || rk / S == hy)) {
+        tot[rk] = cluster.map_shared_rank(scal, unsigned(rk))[0];
+        uu[rk] = cluster.map_shared_rank(u_s, unsigned(rk))[tid];
+        qq[rk] = cluster.map_shared_rank(qsum_s, unsigned(rk))[tid];
+      }
+    }
+    auto head_probe = [&](int y) {
+      float t = 0.f, u2 = 0.f, q2 = 0.f;
+#pragma unroll
+      for (int rk = 0; rk < kMaxCluster; ++rk)
+        if (rk >= y * S && rk < (y + 1) * S) { t += tot[rk]; u2 += uu[rk]; q2 += qq[rk]; }
+      return t > 0.f ? u2 / t : q2 / float(W);      // all-zero bias: uniform weights
+    };
+    p.probe_qh[hd + tid] = head_probe(cy > 1 ? hy : 0);
+    if (hy == 0) {
+      float acc = 0.f;
+      for (int y = 0; y < p.group; ++y) acc += head_probe(y);
+      p.probe_kv[(size_t(unit) * p.n_kv_heads + h / p.group) * D + tid] = acc / float(p.group);
+    }
+  }
+  cluster.sync();      // peers keep their shared memory alive until the leaders have read it
 }
 
-// G = 1 (or no cluster): KV probe is the query-head probe.
-__global__ void copy_probe_kernel(const float* src, float* dst, size_t n) {
-  size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x;
-  if (i < n) dst[i] = src[i];
+template <typename T, int D>
+int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaStream_t st) {
+  const int W = p.n_tokens;
+  const int cy = p.do_probe ? p.group : 1;
+  auto kern = bias_probe_kernel<T, D>;
+  constexpr int VN = Vec16<T>::N;
+  constexpr int RL = kThreads / (D / VN), NP = kThreads / D;
+  // Clusters stay within the portable size of 8: 16-CTA clusters were measured slower here (they
+  // are scheduled one GPC at a time and their barrier costs more than the extra SMs bring).
+  for (int max_cluster = 8; max_cluster >= 8; max_cluster >>= 1) {
+    int split = max_cluster / cy;
+    if (split < 1) split = 1;
+    while (split > 1 && (W + split - 1) / split < 32) split >>= 1;
+    p.split = split;
+    p.rows_per_cta = (W + split - 1) / split;
+    const size_t tile_bytes = (size_t(p.rows_per_cta) * D * sizeof(T) + 127) & ~size_t(127);
+    const size_t smem = tile_bytes + sizeof(float) * (size_t(2) * RL * D + 2 * NP * D + 6 * D + 4 + 32 +
+                                                       ((p.rows_per_cta + 3) & ~3)) + 16;
+    if (smem > 220 * 1024) return ACTQKV_ERR_SHAPE;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+      return ACTQKV_ERR_LAUNCH;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(split, cfg->n_q_heads, b.units());
+    lc.blockDim = dim3(kThreads, 1, 1);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = split;
+    attr[0].val.clusterDim.y = cy;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lc, kern, p) == cudaSuccess) return launch_status();
+    (void)cudaGetLastError();
+  }
+  return ACTQKV_ERR_LAUNCH;
 }
 
 template <typename T>
 int launch(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaStream_t st) {
-  const int D = cfg->head_dim, W = p.n_tokens;
-  const size_t tile_bytes = (size_t(W) * D * sizeof(T) + 15) & ~size_t(15);
-  const size_t smem = tile_bytes + sizeof(float) * (size_t(kThreads / D) * D + 3 * D + 32 + W);
-  if (smem > 200 * 1024) return ACTQKV_ERR_SHAPE;
-  const bool cluster = p.do_probe && p.group > 1;
-  auto kern = cluster ? bias_probe_kernel<T, true> : bias_probe_kernel<T, false>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-    return ACTQKV_ERR_LAUNCH;
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(cfg->n_q_heads, b.units(), 1);
-  lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = smem;
-  lc.stream = st;
-  cudaLaunchAttribute attr[1];
-  if (cluster) {
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = p.group;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-  }
-  if (cudaLaunchKernelEx(&lc, kern, p) != cudaSuccess) return ACTQKV_ERR_LAUNCH;
-  if (p.do_probe && p.group == 1) {
-    const size_t n = size_t(b.units()) * cfg->n_q_heads * D;
-    copy_probe_kernel<<<unsigned((n + 255) / 256), 256, 0, st>>>(p.probe_qh, p.probe_kv, n);
-  }
-  return launch_status();
+  return cfg->head_dim == 64 ? launch_d<T, 64>(cfg, b, p, st) : launch_d<T, 128>(cfg, b, p, st);
 }
 
 int run(const actqkv_config* cfg, const actqkv_batch* batch, BiasProbeParams& p, void* stream) {
