@@ -206,7 +206,7 @@ def run_ours(args):
             else:
                 fn()
 
-    launches_per_step = 6   # bias_probe, score, cut-off chain, select, attention, append
+    launches_per_step = 5   # bias_probe, score, cut-off + select, attention, append
 
     def barrier():
         if world > 1:

@@ -2,7 +2,7 @@
 //
 // One launch, two roles selected by blockIdx.x:
 //   copy CTAs   scatter the step's K / V rows into their pages (16-byte vectors);
-//   repr CTAs   one per (completed block, KV head): each of the r representatives is the
+//   repr CTAs   one per (completed block, KV head, representative): each representative is the
 //               mean of B/r consecutive keys, read as 16-byte vectors by all threads at once
 //               and accumulated in fp64 (exact for bf16 inputs, so the rounded table is
 //               bit-reproducible), rounded to the cache dtype; the inverse norm is taken from
@@ -66,9 +66,10 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
     return;
   }
 
-  // ---- repr role: one CTA per (completed block, KV head)
+  // ---- repr role: one CTA per (completed block, KV head, representative)
   const int rid = blockIdx.x - p.copy_ctas;
-  const int g = rid % p.n_kv_heads, nb = rid / p.n_kv_heads;
+  const int i = rid % p.n_repr;
+  const int g = (rid / p.n_repr) % p.n_kv_heads, nb = rid / (p.n_repr * p.n_kv_heads);
   const int64_t p1 = p0 + p.n_tokens;
   const int64_t done0 = p0 > p.n_init ? (p0 - p.n_init) / p.block : 0;
   const int64_t done1 = p1 > p.n_init ? (p1 - p.n_init) / p.block : 0;
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
   const size_t row0 = ((size_t(unit) * p.n_kv_heads + g) * p.n_cap + size_t(b)) * p.n_repr;
   T* tab = static_cast<T*>(p.repr_k) + row0 * D;
   const int64_t blk0 = int64_t(p.n_init) + b * p.block;
-  for (int i = 0; i < p.n_repr; ++i) {
+  {
     const int lo = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? i * seg : i * seg + seg / 2;
     const int hi = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? (i + 1) * seg : lo + 1;
     double acc[VN];
@@ -130,10 +131,11 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
       sq_s[tid] = stored * stored;
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid < 32) {                       // fixed order: lane partial sums, then a shuffle tree
       float t = 0.f;
-      for (int cc = 0; cc < D; ++cc) t += sq_s[cc];
-      p.repr_inv_norm[row0 + i] = t > 0.f ? rsqrtf(t) : 0.f;
+      for (int cc = tid; cc < D; cc += 32) t += sq_s[cc];
+      t = warp_sum(t);
+      if (tid == 0) p.repr_inv_norm[row0 + i] = t > 0.f ? rsqrtf(t) : 0.f;
     }
   }
 }
@@ -166,7 +168,7 @@ extern "C" int actqkv_append_window(const actqkv_config* cfg, const actqkv_batch
   const int64_t vecs = int64_t(n_tokens) * cfg->n_kv_heads * vpr;
   p.copy_ctas = int(std::min<int64_t>((vecs + kThreads - 1) / kThreads, 296));
   p.max_new_blocks = n_tokens / cfg->block + 2;
-  dim3 grid(p.copy_ctas + p.max_new_blocks * cfg->n_kv_heads, b.units());
+  dim3 grid(p.copy_ctas + p.max_new_blocks * cfg->n_kv_heads * cfg->n_repr, b.units());
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const size_t smem = sizeof(double) * size_t(kThreads / vpr) * cfg->head_dim + sizeof(float) * cfg->head_dim;
   if (cfg->dtype == ACTQKV_BF16) append_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(p);

@@ -1,6 +1,6 @@
 // Step 4: dynamic KV cut-off (Eq. 12) and top-c block selection (Algorithm 1, last loop).
 //
-// Two kernels, no host round trip:
+// No host round trip.  A call that batches several layers runs two kernels:
 //   cutoff_chain_kernel  one CTA per sequence.  Warps evaluate (or read) the per-head
 //                        information densities of every batched layer, then one thread walks
 //                        the layers shallow -> deep in fp64: B^l from Eq. 12, the granted
@@ -9,8 +9,16 @@
 //                        keys in shared memory; an MSB-first 8-bit radix select finds the c-th
 //                        largest key; equal keys are admitted lowest index first; the survivors
 //                        are compacted in ascending block order with block-wide scans.
+// A call for one layer (the usual layer-by-layer use) runs select_kernel alone: the Hkv CTAs of a
+// sequence form a thread-block cluster, each takes its head's density, they exchange the values
+// through distributed shared memory, every CTA evaluates Eq. 12 for itself and the first one
+// writes the budget state back.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "stages.cuh"
+
+namespace cg = cooperative_groups;
 
 using namespace actqkv;
 
@@ -30,6 +38,19 @@ struct ChainParams {
   int n_kv_heads, n_cap, L, Lb, layer0, k_blocks, cap_blocks, thetabar_mode;
   float beta;
 };
+
+// Eq. 12 for one layer with n > 0 candidates: returns the granted count c and the un-rounded
+// budget; `rest` = sum over the deeper layers of their mean density (theta-bar).
+struct Grant { int c; double real; };
+__device__ __forceinline__ Grant grant_layer(double th, double rest, double b_rem, int layers_left, int n, int cap) {
+  Grant gr;
+  const double den = th + rest;
+  gr.real = den > 0.0 ? th / den * b_rem : b_rem / double(layers_left);
+  const double fl = floor(gr.real + 0.5);
+  int c = fl > 2.0e9 ? 2000000000 : (fl < -2.0e9 ? -2000000000 : int(fl));
+  gr.c = max(min(1, n), min(c, min(cap, n)));
+  return gr;
+}
 
 __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams p) {
   extern __shared__ float theta_h[];   // [Lb][Hkv]
@@ -63,8 +84,7 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
     const int layer = p.layer0 + l;
     if (layer == 0) b_rem = double(p.L) * double(p.k_blocks);
     const double th = layer_theta(l);
-    int c = 0;
-    double real = 0.0;
+    Grant gr{0, 0.0};
     if (n > 0) {
       double rest = 0.0;
       for (int j = layer + 1; j < p.L; ++j) {
@@ -76,18 +96,14 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
           rest += th;
         }
       }
-      const double den = th + rest;
-      real = den > 0.0 ? th / den * b_rem : b_rem / double(p.L - layer);
-      const double fl = floor(real + 0.5);
-      c = fl > 2.0e9 ? 2000000000 : (fl < -2.0e9 ? -2000000000 : int(fl));
-      c = max(min(1, n), min(c, min(p.cap_blocks, n)));
-      b_rem -= double(c);
+      gr = grant_layer(th, rest, b_rem, p.L - layer, n, p.cap_blocks);
+      b_rem -= double(gr.c);
       hist_sum[layer] += th;
       hist_cnt[layer] += 1.0;
     }
     const size_t unit = size_t(seq) * p.Lb + l;
-    p.sel_count[unit] = c;
-    if (p.budget_real) p.budget_real[unit] = float(real);
+    p.sel_count[unit] = gr.c;
+    if (p.budget_real) p.budget_real[unit] = float(gr.real);
   }
   st[0] = b_rem;
 }
@@ -122,103 +138,170 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* t
   return base + inc - v;
 }
 
+// kFused: the call holds one layer; the grid is launched as clusters of n_kv_heads CTAs (one
+// sequence each) and the cut-off chain of that layer is evaluated here (ch), else sel_count is
+// an input written by cutoff_chain_kernel.
+template <bool kFused>
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_cand,
-              const int32_t* __restrict__ sel_count, int32_t* __restrict__ sel_idx, int n_kv_heads,
-              int n_cap, int cap_blocks, int n_layers, int32_t* status) {
+              int32_t* __restrict__ sel_count, int32_t* __restrict__ sel_idx, int n_kv_heads,
+              int n_cap, int cap_blocks, int n_layers, int32_t* status, ChainParams ch) {
   extern __shared__ uint32_t keys[];           // [n_cap]
   __shared__ int hist[256];
   __shared__ int warp_tot[kSelThreads / 32];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_need;
+  __shared__ float sh_theta;                   // this head's density (read by the cluster peers)
+  __shared__ int sh_count;
   const int g = blockIdx.x, unit = blockIdx.y, tid = threadIdx.x;
   const int n = min(n_cand[unit / n_layers], n_cap);
-  int c = sel_count[unit];
-  if (c < 0 || c > min(cap_blocks, n)) {
-    if (tid == 0) set_status(status, ACTQKV_DEV_BAD_SELECTION);
-    c = max(0, min(c, min(cap_blocks, n)));
+  const float* s = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
+  int c;
+  if constexpr (kFused) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int seq = unit;                      // one layer per call: unit == sequence
+    const int layer = ch.layer0;
+    double* st = ch.state + size_t(seq) * (1 + 2 * ch.L);
+    // the old state is read by every CTA before the cluster barrier, written by CTA 0 after it
+    double b_rem = 0.0, rest_hist = 0.0;
+    int no_hist = 0;
+    if (tid == 0) {
+      b_rem = layer == 0 ? double(ch.L) * double(ch.k_blocks) : st[0];
+      for (int j = layer + 1; j < ch.L; ++j) {
+        const double cnt = st[1 + ch.L + j];
+        if (cnt > 0.0) rest_hist += st[1 + j] / cnt; else ++no_hist;
+      }
+    }
+    if (tid < 32) {
+      const size_t uh = size_t(unit) * n_kv_heads + g;
+      float th;
+      if (ch.theta_in) {
+        th = ch.theta_in[uh];
+      } else {
+        th = warp_entropy(s, n, ch.beta);
+        if (tid == 0 && ch.theta_out) ch.theta_out[uh] = th;
+      }
+      if (tid == 0) sh_theta = th;
+    }
+    cluster.sync();
+    if (tid == 0) {
+      float th_h[8];                             // all peers' values first: independent remote loads
+#pragma unroll
+      for (int h2 = 0; h2 < 8; ++h2)
+        th_h[h2] = h2 < n_kv_heads ? *cluster.map_shared_rank(&sh_theta, unsigned(h2)) : 0.f;
+      double sum = 0.0;
+#pragma unroll
+      for (int h2 = 0; h2 < 8; ++h2) sum += double(th_h[h2]);
+      const double th = sum / double(n_kv_heads);
+      Grant gr{0, 0.0};
+      if (n > 0) {
+        // layers without history count with this layer's density; with every layer in the call
+        // (L == 1) there is no deeper layer and both theta-bar readings coincide
+        const double rest = rest_hist + double(no_hist) * th;
+        gr = grant_layer(th, rest, b_rem, ch.L - layer, n, ch.cap_blocks);
+        if (g == 0) {
+          st[0] = b_rem - double(gr.c);
+          st[1 + layer] += th;
+          st[1 + ch.L + layer] += 1.0;
+        }
+      } else if (g == 0) {
+        st[0] = b_rem;
+      }
+      if (g == 0) {
+        sel_count[unit] = gr.c;
+        if (ch.budget_real) ch.budget_real[unit] = float(gr.real);
+      }
+      sh_count = gr.c;
+    }
+    __syncthreads();
+    c = sh_count;
+  } else {
+    c = sel_count[unit];
+    if (c < 0 || c > min(cap_blocks, n)) {
+      if (tid == 0) set_status(status, ACTQKV_DEV_BAD_SELECTION);
+      c = max(0, min(c, min(cap_blocks, n)));
+    }
   }
   int32_t* out = sel_idx + (size_t(unit) * n_kv_heads + g) * cap_blocks;
   for (int i = c + tid; i < cap_blocks; i += kSelThreads) out[i] = -1;
-  if (c == 0) return;
   if (c >= n) {
-    for (int i = tid; i < n; i += kSelThreads) out[i] = i;
-    return;
-  }
-  const float* s = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
-  for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i]);
-  if (tid == 0) { sh_prefix = 0u; sh_need = c; }
-  __syncthreads();
+    for (int i = tid; i < min(n, c); i += kSelThreads) out[i] = i;
+  } else if (c > 0) {
+    for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i]);
+    if (tid == 0) { sh_prefix = 0u; sh_need = c; }
+    __syncthreads();
 
-  // ---- radix select of the c-th largest key
-  uint32_t mask = 0u;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    hist[tid] = 0;                                        // kSelThreads == 256 bins
-    __syncthreads();
-    const uint32_t prefix = sh_prefix;
-    for (int i = tid; i < n; i += kSelThreads) {
-      const uint32_t k = keys[i];
-      if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // lane l owns bins 255-8l .. 248-8l (descending)
-      int loc[8], sum = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { loc[j] = hist[255 - 8 * tid - j]; sum += loc[j]; }
-      int inc = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, inc, o);
-        if (tid >= o) inc += t;
+    // ---- radix select of the c-th largest key
+    uint32_t mask = 0u;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      hist[tid] = 0;                                        // kSelThreads == 256 bins
+      __syncthreads();
+      const uint32_t prefix = sh_prefix;
+      for (int i = tid; i < n; i += kSelThreads) {
+        const uint32_t k = keys[i];
+        if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
       }
-      int before = inc - sum;
-      const int need = sh_need;
-      if (before < need && need <= inc) {
+      __syncthreads();
+      if (tid < 32) {
+        // lane l owns bins 255-8l .. 248-8l (descending)
+        int loc[8], sum = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (before < need && need <= before + loc[j]) {
-            sh_prefix = prefix | (uint32_t(255 - 8 * tid - j) << shift);
-            sh_need = need - before;
-            before = need;                                  // stop further matches
-          } else {
-            before += loc[j];
+        for (int j = 0; j < 8; ++j) { loc[j] = hist[255 - 8 * tid - j]; sum += loc[j]; }
+        int inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (tid >= o) inc += t;
+        }
+        int before = inc - sum;
+        const int need = sh_need;
+        if (before < need && need <= inc) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (before < need && need <= before + loc[j]) {
+              sh_prefix = prefix | (uint32_t(255 - 8 * tid - j) << shift);
+              sh_need = need - before;
+              before = need;                                  // stop further matches
+            } else {
+              before += loc[j];
+            }
           }
         }
       }
+      mask |= 255u << shift;
+      __syncthreads();
     }
-    mask |= 255u << shift;
-    __syncthreads();
-  }
-  const uint32_t thr = sh_prefix;
-  const int need_eq = sh_need;          // how many keys equal to thr are admitted (>= 1)
+    const uint32_t thr = sh_prefix;
+    const int need_eq = sh_need;          // how many keys equal to thr are admitted (>= 1)
 
-  // ---- admit equal keys lowest index first, compact ascending
-  const int per = (n + kSelThreads - 1) / kSelThreads;
-  const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
-  int eq = 0;
-  for (int i = i0; i < i1; ++i) eq += keys[i] == thr;
-  int tot;
-  int eq_before = block_exclusive_scan(eq, warp_tot, &tot);
-  int cnt = 0;
-  {
-    int e = eq_before;
-    for (int i = i0; i < i1; ++i) {
-      const uint32_t k = keys[i];
-      if (k > thr) ++cnt;
-      else if (k == thr) { if (e < need_eq) ++cnt; ++e; }
+    // ---- admit equal keys lowest index first, compact ascending
+    const int per = (n + kSelThreads - 1) / kSelThreads;
+    const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
+    int eq = 0;
+    for (int i = i0; i < i1; ++i) eq += keys[i] == thr;
+    int tot;
+    int eq_before = block_exclusive_scan(eq, warp_tot, &tot);
+    int cnt = 0;
+    {
+      int e = eq_before;
+      for (int i = i0; i < i1; ++i) {
+        const uint32_t k = keys[i];
+        if (k > thr) ++cnt;
+        else if (k == thr) { if (e < need_eq) ++cnt; ++e; }
+      }
+    }
+    int pos = block_exclusive_scan(cnt, warp_tot, &tot);
+    {
+      int e = eq_before;
+      for (int i = i0; i < i1; ++i) {
+        const uint32_t k = keys[i];
+        bool take = k > thr;
+        if (k == thr) { take = e < need_eq; ++e; }
+        if (take && pos < cap_blocks) out[pos++] = i;
+      }
     }
   }
-  int pos = block_exclusive_scan(cnt, warp_tot, &tot);
-  {
-    int e = eq_before;
-    for (int i = i0; i < i1; ++i) {
-      const uint32_t k = keys[i];
-      bool take = k > thr;
-      if (k == thr) { take = e < need_eq; ++e; }
-      if (take && pos < cap_blocks) out[pos++] = i;
-    }
-  }
+  if constexpr (kFused) cg::this_cluster().sync();   // peers may still be reading sh_theta
 }
 
 int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores, const float* theta_in,
@@ -234,17 +317,34 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
   p.n_kv_heads = cfg->n_kv_heads; p.n_cap = cfg->n_cap; p.L = cfg->n_layers; p.Lb = b.n_layers;
   p.layer0 = b.layer0; p.k_blocks = cfg->k_blocks; p.cap_blocks = cfg->cap_blocks;
   p.thetabar_mode = cfg->thetabar_mode; p.beta = cfg->beta;
-  const size_t sm_chain = sizeof(float) * size_t(b.n_layers) * cfg->n_kv_heads;
-  if (sm_chain > 48 * 1024) return ACTQKV_ERR_SHAPE;
-  cutoff_chain_kernel<<<b.n_seq, kChainThreads, sm_chain, st>>>(p);
-  if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;
-  if (cfg->cap_blocks == 0) return ACTQKV_OK;
   const size_t sm_sel = size_t(cfg->n_cap) * 4;
-  if (sm_sel > 48 * 1024 &&
-      cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sm_sel)) != cudaSuccess)
+  const bool fused = b.n_layers == 1 && cfg->n_kv_heads <= 8 && cfg->cap_blocks > 0;
+  auto kern = fused ? select_kernel<true> : select_kernel<false>;
+  if (sm_sel > 40 * 1024 &&
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sm_sel)) != cudaSuccess)
     return ACTQKV_ERR_LAUNCH;
-  select_kernel<<<dim3(cfg->n_kv_heads, b.units()), kSelThreads, sm_sel, st>>>(
-      scores, n_cand, sel_count, sel_idx, cfg->n_kv_heads, cfg->n_cap, cfg->cap_blocks, b.n_layers, status);
+  if (!fused) {
+    const size_t sm_chain = sizeof(float) * size_t(b.n_layers) * cfg->n_kv_heads;
+    if (sm_chain > 48 * 1024) return ACTQKV_ERR_SHAPE;
+    cutoff_chain_kernel<<<b.n_seq, kChainThreads, sm_chain, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;
+    if (cfg->cap_blocks == 0) return ACTQKV_OK;
+  }
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(cfg->n_kv_heads, b.units(), 1);
+  lc.blockDim = dim3(kSelThreads, 1, 1);
+  lc.dynamicSmemBytes = sm_sel;
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = fused ? cfg->n_kv_heads : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  if (cudaLaunchKernelEx(&lc, kern, scores, n_cand, sel_count, sel_idx, cfg->n_kv_heads, cfg->n_cap,
+                         cfg->cap_blocks, b.n_layers, status, p) != cudaSuccess)
+    return ACTQKV_ERR_LAUNCH;
   return launch_status();
 }
 
