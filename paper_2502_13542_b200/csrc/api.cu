@@ -54,9 +54,12 @@ extern "C" int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv
   a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
   a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  // ACTQKV_ATTENTION=simt forces the general kernel (debugging aid; the default picks by shape).
+  // ACTQKV_ATTENTION=simt forces the general kernel, =tc1 the single-CTA tensor-core kernel
+  // (debugging aids; the default picks by shape).
   const char* force = std::getenv("ACTQKV_ATTENTION");
   const bool simt_only = force && std::strcmp(force, "simt") == 0;
+  const bool tc1_only = force && std::strcmp(force, "tc1") == 0;
+  if (!simt_only && !tc1_only && attention_tc2_supported(cfg, n_tokens)) return launch_attention_tc2(cfg, b, a, st);
   if (!simt_only && attention_tc_supported(cfg, n_tokens)) return launch_attention_tc(cfg, b, a, st);
   return launch_attention_simt(cfg, b, a, st);
 }

@@ -42,5 +42,8 @@ struct AttnArgs {
 int launch_attention_simt(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 bool attention_tc_supported(const actqkv_config* cfg, int n_tokens);
 int launch_attention_tc(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
+// The same kernel for pairs of CTAs sharing each K / V tile (needs an even number of query heads per KV head).
+bool attention_tc2_supported(const actqkv_config* cfg, int n_tokens);
+int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 
 }  // namespace actqkv

@@ -265,11 +265,13 @@ def test_edge_cases_and_errors(B):
     assert int(st4.status.item()) == 0
 
 
+@pytest.mark.parametrize("kernel", ["pair", "tc1"])
 @pytest.mark.parametrize("target", [1, 3])
-def test_tc_attention_repeatable_and_matches_general_kernel(B, monkeypatch, target):
-    """The tensor-core attention is run many times on the same state: every run must give the
-    same bits (no timing dependence), and agree with the general fp32 kernel.  Window 1 gives
-    the shortest key-tile loops (5 to 8 tiles), window 3 longer ones."""
+def test_tc_attention_repeatable_and_matches_general_kernel(B, monkeypatch, target, kernel):
+    """The tensor-core attention (the CTA-pair kernel the shape selects by default, and the
+    single-CTA kernel) is run many times on the same state: every run must give the same bits
+    (no timing dependence), and agree with the general fp32 kernel.  Window 1 gives the shortest
+    key-tile loops (5 to 8 tiles), window 3 longer ones."""
     import torch
     spec = wl.llama3_8b_layer().replace(context=4096)
     cfg = B.make_config(spec, out_dtype=B.F32)
@@ -295,6 +297,8 @@ def test_tc_attention_repeatable_and_matches_general_kernel(B, monkeypatch, targ
     attend(gen)
     torch.cuda.synchronize()
     monkeypatch.delenv("ACTQKV_ATTENTION")
+    if kernel == "tc1":
+        monkeypatch.setenv("ACTQKV_ATTENTION", "tc1")
     outs = [torch.zeros_like(out) for _ in range(8)]
     ref = None
     for rep in range(60):
