@@ -18,7 +18,7 @@
 // A query row (= TMEM lane) is shared by two softmax threads, one per column half; they
 // exchange their half-row maxima through shared memory once per tile.  Running max / sum are
 // kept in base 2; P is written back over the S columns as two bf16 terms (hi + lo); O is
-// rescaled in TMEM only when a row's max grew by more than 2^8 (lazy rescale).
+// rescaled in TMEM only when a row's max grew by more than 2^32 (lazy rescale).
 //
 // TMEM columns: S/P buffers 0..2 at [0,128) [128,256) [256,384), O at [384,512).
 // S = Q K^T uses both operands from shared memory (K-major, SW128); O += P V takes P from
@@ -162,10 +162,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     int issued = 0;
     for (int j = 0; j < n_tiles && ok; ++j) {
       const int s = j % kRing, it = j / kRing;
-      if ((j & 3) == 0) {
-        page_cur = page_next;
-        page_next = resolve((j >> 2) + 1);
-      }
+      if ((j & 3) == 0) page_cur = page_next;
       const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + slot);
       if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -180,6 +177,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tma_load_3d(sbase + lane * kSubTileBytes, tm_win, full, lane * 64, g, unit * nt + (j - past_tiles) * kBN);
       }
       issued = j + 1;
+      if ((j & 3) == 0) page_next = resolve((j >> 2) + 1);   // after the issue: its stall is behind the ring
     }
     // drain: every issued copy must have landed before the CTA may exit on the abort path
     if (!ok) {
@@ -273,12 +271,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           mx = max3(mx, x0, x1);
         }
       } else {
+        float mx3 = -INFINITY, mx4 = -INFINITY;           // four independent chains
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
+        for (int i = 0; i < 32; i += 4) {
           mx = max3(mx, lo2(sv[i]), hi2(sv[i]));
           mx2 = max3(mx2, lo2(sv[i + 1]), hi2(sv[i + 1]));
+          mx3 = max3(mx3, lo2(sv[i + 2]), hi2(sv[i + 2]));
+          mx4 = max3(mx4, lo2(sv[i + 3]), hi2(sv[i + 3]));
         }
-        mx = fmaxf(mx, mx2);
+        mx = fmaxf(max3(mx, mx2, mx3), mx4);
       }
       // the row's maximum over both column halves
       float* xrow = xchg + (j & 1) * 256 + row;

@@ -79,17 +79,21 @@ __device__ __forceinline__ void tc2_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"(both) : "memory");
 }
-__device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+// Descriptors are passed as (low, high) words; kAcc = accumulate into D (else overwrite).
+template <bool kAcc>
+__device__ __forceinline__ void mma2_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "n"(kAcc ? 1 : 0) : "memory");
 }
-__device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -212,10 +216,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     int issued = 0;
     for (int j = 0; j < n_tiles && ok; ++j) {
       const int s = j % kRing, it = j / kRing;
-      if ((j & 3) == 0) {
-        page_cur = page_next;
-        page_next = resolve((j >> 2) + 1);
-      }
+      if ((j & 3) == 0) page_cur = page_next;
       const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + my_granule);
       if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -239,6 +240,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
       }
       issued = j + 1;
+      if ((j & 3) == 0) page_next = resolve((j >> 2) + 1);   // after the issue: its stall is behind the ring
     }
     // drain: what this CTA issued must have landed before it may leave on the abort path; its
     // copies complete on the leader's barriers, which only the leader can poll, so the peer waits
@@ -260,50 +262,69 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       constexpr uint32_t idesc_qk = make_idesc(false, 2 * kBM, kBN);
       constexpr uint32_t idesc_pv = make_idesc(true, 2 * kBM, kBN);
       const uint32_t tmem_o = tmem + kSBuf * 128;
+      // operand descriptors: high words are constants, low words advance by constant steps
+      constexpr uint32_t kHi = desc_hi(1024u);
+      const uint32_t q_lo = desc_lo(q_smem, 16u);
       bool ok = mbar_wait(bar_q, 0, abort_flag);
-      auto issue_qk = [&](int j) {
+      auto issue_qk = [&](int j) {                 // K(j) has landed
         const int s = j % kRing;
-        ok = ok && mbar_wait(bar_kfull(s), (j / kRing) & 1, abort_flag);
-        if (!ok) return;
         tc_fence_after();
-        const uint32_t kbase = k_ring + s * kHalfBytes;
+        const uint32_t k_lo = desc_lo(k_ring + s * kHalfBytes, 16u);
         const uint32_t s_tmem = tmem + (j % kSBuf) * 128;
+        // A: this CTA's 128 query rows; B: this CTA's 64 keys; both advance 16 channels per step
+        mma2_ss<false>(s_tmem, q_lo, k_lo, kHi, idesc_qk);
 #pragma unroll
-        for (int k = 0; k < kD / 16; ++k) {
-          // A: this CTA's 128 query rows; B: this CTA's 64 keys; both advance 16 channels per step
-          const uint32_t a_off = (k >> 2) * kSubTileBytes + (k & 3) * 32u;
-          const uint32_t b_off = (k >> 2) * kKSubBytes + (k & 3) * 32u;
-          mma2_ss(s_tmem, make_desc(q_smem + a_off, 16u, 1024u), make_desc(kbase + b_off, 16u, 1024u), idesc_qk,
-                  k > 0 ? 1u : 0u);
+        for (int k = 1; k < kD / 16; ++k) {
+          constexpr uint32_t kUnit = 16;     // descriptor addresses count 16-byte units
+          const uint32_t a_off = ((k >> 2) * kSubTileBytes + (k & 3) * 32u) / kUnit;
+          const uint32_t b_off = ((k >> 2) * kKSubBytes + (k & 3) * 32u) / kUnit;
+          mma2_ss<true>(s_tmem, q_lo + a_off, k_lo + b_off, kHi, idesc_qk);
         }
         tc2_commit(bar_kempty(s));
         tc2_commit(bar_sfull(j % kSBuf));
       };
-      auto issue_pv = [&](int i) {
+      auto issue_pv = [&](int i) {                 // V(i) has landed and both CTAs published P(i)
         const int s = i % kRing, b = i % kSBuf;
-        ok = ok && mbar_wait(bar_vfull(s), (i / kRing) & 1, abort_flag);
-        ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag);
-        if (!ok) return;
         tc_fence_after();
-        const uint32_t vbase = v_ring + s * kHalfBytes;
+        const uint32_t v_lo = desc_lo(v_ring + s * kHalfBytes, kSubTileBytes);
         const uint32_t p_tmem = tmem + b * 128;
 #pragma unroll
         for (int k = 0; k < kBN / 16; ++k) {
           // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
           // term, then the 8 columns of the lo term of the same keys against the same V rows.
-          const uint64_t bdesc = make_desc(vbase + k * 2048u, kSubTileBytes, 1024u);
+          const uint32_t b_lo = v_lo + k * (2048u / 16u);
           const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
-          mma2_ts(tmem_o, pa, bdesc, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
-          mma2_ts(tmem_o, pa + 16, bdesc, idesc_pv, 1u);
+          mma2_ts(tmem_o, pa, b_lo, kHi, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
+          mma2_ts(tmem_o, pa + 16, b_lo, kHi, idesc_pv, 1u);
         }
         tc2_commit(bar_vempty(s));
         tc2_commit(bar_pvdone(i % kPvRing));
       };
-      issue_qk(0);
-      if (n_tiles > 1) issue_qk(1);
-      for (int i = 0; i < n_tiles && ok; ++i) {
-        if (i + 2 < n_tiles) issue_qk(i + 2);
-        issue_pv(i);
+      // Whichever product has its operands is issued next: S = Q K^T may run up to kSBuf tiles
+      // ahead of O += P V (QK(j) reuses the buffer PV(j - kSBuf) read, and the pipe executes in
+      // issue order), so a late K tile does not hold back a ready P V, nor the reverse.
+      int qk = 0, pv = 0;
+      uint32_t idle = 0;
+      while (pv < n_tiles && ok) {
+        bool progressed = false;
+        const bool qk_allowed = qk < n_tiles && qk < pv + kSBuf;
+        if (qk_allowed && mbar_try_wait(bar_kfull(qk % kRing), (qk / kRing) & 1)) {
+          issue_qk(qk);
+          ++qk;
+          progressed = true;
+        }
+        if (pv < qk && mbar_try_wait(bar_vfull(pv % kRing), (pv / kRing) & 1) &&
+            mbar_try_wait(bar_pfull(pv % kSBuf), (pv / kSBuf) & 1)) {
+          issue_pv(pv);
+          ++pv;
+          progressed = true;
+        }
+        if (progressed) {
+          idle = 0;
+        } else if (++idle >= kSpinLimit || ((idle & 1023u) == 0 && *abort_flag)) {
+          *abort_flag = 1;
+          ok = false;
+        }
       }
       if (ok) tc2_commit(bar_done);
     }
@@ -340,12 +361,15 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           mx = max3(mx, x0, x1);
         }
       } else {
+        float mx3 = -INFINITY, mx4 = -INFINITY;           // four independent chains
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
+        for (int i = 0; i < 32; i += 4) {
           mx = max3(mx, lo2(sv[i]), hi2(sv[i]));
           mx2 = max3(mx2, lo2(sv[i + 1]), hi2(sv[i + 1]));
+          mx3 = max3(mx3, lo2(sv[i + 2]), hi2(sv[i + 2]));
+          mx4 = max3(mx4, lo2(sv[i + 3]), hi2(sv[i + 3]));
         }
-        mx = fmaxf(mx, mx2);
+        mx = fmaxf(max3(mx, mx2, mx3), mx4);
       }
       // the row's maximum over both column halves
       float* xrow = xchg + (j & 1) * 256 + row;

@@ -11,7 +11,9 @@ namespace actqkv {
 namespace tc {
 
 constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr float kRescaleThreshold = 8.0f;                // log2 units
+// O is rescaled only when a row's maximum grew by more than this (log2 units).  P = 2^(x - m) may
+// then reach 2^32: bf16 and fp32 have the range, and the relative precision does not change.
+constexpr float kRescaleThreshold = 32.0f;
 
 struct TcParams {
   AttnArgs a;
@@ -157,6 +159,14 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= uint64_t(1) << 46;        // descriptor version
   d |= uint64_t(2) << 61;        // SWIZZLE_128B
   return d;
+}
+// The same descriptor as two 32-bit words, so that the issuing thread advances an operand with one
+// 32-bit add on the low word (start address in 16-byte units, no carry into the other fields).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);   // SBO, version 1, SWIZZLE_128B
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M x N tile (M = 256 for a CTA pair).
 __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, int m, int n) {
