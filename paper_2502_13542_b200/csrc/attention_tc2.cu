@@ -16,7 +16,7 @@
 // CTA (cluster rank 0) issues MMAs.  Cross-CTA signalling:
 //   TMA loads of both CTAs complete on the LEADER's "full" barriers (cta_group::2 form of the load);
 //   the leader's commits are multicast to the barriers of both CTAs (slot released, S ready, P V done);
-//   the softmax threads of both CTAs arrive on the leader's "P ready" barrier (512 arrivals).
+//   the softmax warps of both CTAs arrive on the leader's "P ready" barrier (one arrival per warp).
 // TMEM columns (both CTAs alike): S/P buffers 0..2 at [0,128) [128,256) [256,384), O at [384,512).
 // Every wait on an mbarrier is bounded; on expiry the CTA flags ACTQKV_DEV_TIMEOUT, stops issuing
 // work and drains; both CTAs meet at a cluster barrier before they free their TMEM.
@@ -167,7 +167,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
       mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
     }
-    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 512); }
+    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 16); }
     for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
     mbar_init(bar_done, 1);
     *abort_flag = 0;
@@ -422,7 +422,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       l += lo2(sum_a) + hi2(sum_a);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive_cluster(leader_addr(bar_pfull(sb)));
+      __syncwarp();                                       // one arrival per warp: 8 warps in each CTA
+      if (lane == 0) mbar_arrive_cluster(leader_addr(bar_pfull(sb)));
     }
     // ---- epilogue: the row sum over both column halves, then this thread's 64 channels of O / l
     ok = ok && mbar_wait(bar_done, 0, abort_flag);

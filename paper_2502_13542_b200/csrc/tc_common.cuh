@@ -148,6 +148,32 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       : "=l"(r[0]), "=l"(r[1]), "=l"(r[2]), "=l"(r[3]), "=l"(r[4]), "=l"(r[5]), "=l"(r[6]), "=l"(r[7]), "=l"(r[8]), "=l"(r[9]), "=l"(r[10]), "=l"(r[11]), "=l"(r[12]), "=l"(r[13]), "=l"(r[14]), "=l"(r[15]), "=l"(r[16]), "=l"(r[17]), "=l"(r[18]), "=l"(r[19]), "=l"(r[20]), "=l"(r[21]), "=l"(r[22]), "=l"(r[23]), "=l"(r[24]), "=l"(r[25]), "=l"(r[26]), "=l"(r[27]), "=l"(r[28]), "=l"(r[29]), "=l"(r[30]), "=l"(r[31]) \
       : "r"(taddr), "r"((taddr) + 32) \
       : "memory")
+// 32 columns as 16 register pairs.
+#define TMEM_LD32P_WAIT(taddr, r) \
+  asm volatile( \
+      "{\n\t.reg .b32 t<32>;\n\t" \
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t0,t1,t2,t3,t4,t5,t6,t7,t8,t9,t10,t11,t12,t13,t14,t15,t16,t17,t18,t19,t20,t21,t22,t23,t24,t25,t26,t27,t28,t29,t30,t31}, [%16];\n\t" \
+      "tcgen05.wait::ld.sync.aligned;\n\t" \
+      "mov.b64 %0, {t0, t1};\n\t" \
+      "mov.b64 %1, {t2, t3};\n\t" \
+      "mov.b64 %2, {t4, t5};\n\t" \
+      "mov.b64 %3, {t6, t7};\n\t" \
+      "mov.b64 %4, {t8, t9};\n\t" \
+      "mov.b64 %5, {t10, t11};\n\t" \
+      "mov.b64 %6, {t12, t13};\n\t" \
+      "mov.b64 %7, {t14, t15};\n\t" \
+      "mov.b64 %8, {t16, t17};\n\t" \
+      "mov.b64 %9, {t18, t19};\n\t" \
+      "mov.b64 %10, {t20, t21};\n\t" \
+      "mov.b64 %11, {t22, t23};\n\t" \
+      "mov.b64 %12, {t24, t25};\n\t" \
+      "mov.b64 %13, {t26, t27};\n\t" \
+      "mov.b64 %14, {t28, t29};\n\t" \
+      "mov.b64 %15, {t30, t31};\n\t" \
+      "}" \
+      : "=l"(r[0]), "=l"(r[1]), "=l"(r[2]), "=l"(r[3]), "=l"(r[4]), "=l"(r[5]), "=l"(r[6]), "=l"(r[7]), "=l"(r[8]), "=l"(r[9]), "=l"(r[10]), "=l"(r[11]), "=l"(r[12]), "=l"(r[13]), "=l"(r[14]), "=l"(r[15]) \
+      : "r"(taddr) \
+      : "memory")
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
@@ -209,18 +235,20 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
-// Barrier between the two softmax warps that share a TMEM lane quadrant (hardware barrier
-// 1 + quadrant, 64 threads; barrier 0 is __syncthreads).  It also ANDs a predicate, so that both
-// take the same decision to go on or to give up.
-__device__ __forceinline__ bool pair_sync_and(int quadrant, bool ok) {
+// Barrier among the kWarps softmax warps that share a TMEM lane quadrant (hardware barrier
+// 1 + quadrant; barrier 0 is __syncthreads).  It also ANDs a predicate, so that all of them take
+// the same decision to go on or to give up.
+template <int kWarps>
+__device__ __forceinline__ bool quadrant_sync_and(int quadrant, bool ok) {
   uint32_t res;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
-      "bar.red.and.pred p, %1, 64, q;\n\t"
+      "bar.red.and.pred p, %1, %3, q;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(res) : "r"(quadrant + 1), "r"(uint32_t(ok)) : "memory");
+      : "=r"(res) : "r"(quadrant + 1), "r"(uint32_t(ok)), "n"(kWarps * 32) : "memory");
   return res != 0;
 }
+__device__ __forceinline__ bool pair_sync_and(int quadrant, bool ok) { return quadrant_sync_and<2>(quadrant, ok); }
 
 // Geometry of the key stream of one CTA, shared by the two producer warps.
 struct KeyStream {
