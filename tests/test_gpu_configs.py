@@ -1,0 +1,216 @@
+"""GPU parity on the larger workload shapes: the 32-layer stack with the budget chain running over
+real scores, the 131072-token sweep, and batched single-token decode with fixed probes.  Every
+intermediate that is cheap for the oracle is compared at every step; attention on stated samples."""
+import numpy as np
+import pytest
+
+from oracle import actqkv_oracle as orc
+from paper_2502_13542_b200 import workloads as wl
+from tests import parity_utils as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2502_13542_b200 import binding
+    return binding
+
+
+def _stack(B, spec, beta, attention_layers, check_windows=None):
+    """All layers of `spec` batched in one call per stage (n_seq = 1, n_layers = L): layer l's
+    budget depends on what the shallower layers were granted (Eq. 12)."""
+    import torch
+    L = spec.n_layers
+    cfg = B.make_config(spec, beta=beta, out_dtype=B.F32)
+    pt = wl.shuffled_page_table(spec, spec.context)
+    st = B.RetrievalState(cfg, n_seq=1, n_layers=L, page_table=pt[None, :])
+    chain = orc.BudgetChain(L, spec.k_blocks, spec.cap_blocks, "streaming")
+    runners = [pu.OracleRunner(spec, layer=l, chain=chain, beta=beta) for l in range(L)]
+    out = torch.zeros(L, spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    counts = []
+    for t in range(spec.n_windows):
+        qs, ks, vs, res = [], [], [], []
+        last = t == spec.n_windows - 1
+        for l in range(L):
+            q = wl.gen_q(spec, l, t)
+            k, v = wl.gen_kv(spec, l, t)
+            qs.append(q); ks.append(k); vs.append(v)
+            res.append(runners[l].step(q, k, v, attention=last and l in attention_layers))
+        st.step(pu.to_device(np.stack(qs), spec), pu.to_device(np.stack(ks), spec),
+                pu.to_device(np.stack(vs), spec), out)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        if check_windows is not None and t not in check_windows:
+            continue
+        got_c = st.sel_count.cpu().numpy().tolist()
+        want_c = [r["c"] for r in res]
+        fragile = [r["fragile"] for r in res]
+        tag = f"{spec.name} beta={beta} window {t}"
+        n = res[0]["n"]
+        if n:
+            for l in range(L):
+                pu.assert_rel(pu.to_numpy(st.scores[l, :, :n]), res[l]["scores"], 1.0, f"{tag} layer {l} scores")
+                pu.assert_rel(pu.to_numpy(st.theta[l]), res[l]["theta"], 1e-30, f"{tag} layer {l} theta")
+        if not any(fragile):
+            assert got_c == want_c, tag
+            for l in range(L):
+                assert pu.compare_selection(pu.to_numpy(st.sel_idx[l]).astype(np.int64), got_c[l], res[l],
+                                            f"{tag} layer {l}") >= 0
+                if last and l in attention_layers:
+                    pu.assert_attention(pu.to_numpy(out[l]), res[l]["out"], f"{tag} layer {l} attention")
+        counts.append((n, want_c))
+    assert abs(float(st.budget_state[0, 0]) - chain.b_rem) < 1e-9
+    return counts
+
+
+def test_tiny_stack32_paper_temperature(B):
+    """32 layers of the tiny shape at beta = 1 (the paper): the densities of the layers are close,
+    the counts stay near k, and they add up to L * k whenever no clamp binds."""
+    spec = wl.tiny_stack32()
+    counts = _stack(B, spec, 1.0, attention_layers={0, 31})
+    unclamped = [c for n, c in counts if n >= spec.cap_blocks and max(c) < spec.cap_blocks]
+    assert unclamped and all(sum(c) == spec.n_layers * spec.k_blocks for c in unclamped)
+    print("tiny stack, beta = 1: per-layer counts at the last window", counts[-1][1])
+
+
+def test_llama_stack32_sharpened_density(B):
+    """32 layers of the LLaMA3-8B shape (bf16, paged) at 16k context with a sharpened softmax
+    (beta = 32) so that the per-layer counts really differ and the cap binds; tensor-core
+    attention of the last window checked on layers 0, 13 and 31."""
+    spec = wl.llama3_8b_stack32().replace(context=16384)
+    counts = _stack(B, spec, 32.0, attention_layers={0, 13, 31}, check_windows=set(range(0, 32, 3)) | {31})
+    late = counts[-1][1]
+    assert len(set(late)) > 2, late
+
+
+def test_long_131k_sweep(B):
+    """131072-token prefill, one layer, cut-off capped at 128 blocks: steps 1-4 and 6 at every
+    window (n grows to 1019 candidate blocks), attention at windows {0, 1, 31, 32, 33, 127, 255}."""
+    import torch
+    spec = wl.long_131k()
+    cfg = B.make_config(spec, out_dtype=B.F32)
+    pt = wl.shuffled_page_table(spec, spec.context)
+    st = B.RetrievalState(cfg, page_table=pt[None, :])
+    run = pu.OracleRunner(spec)
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    att = {0, 1, 31, 32, 33, 127, 255}
+    near = 0
+    for t in range(spec.n_windows):
+        q = wl.gen_q(spec, 0, t)
+        k, v = wl.gen_kv(spec, 0, t)
+        res = run.step(q, k, v, attention=t in att)
+        assert int(st.n_cand.item()) == res["n"]
+        st.step(pu.to_device(q[None], spec), pu.to_device(k[None], spec), pu.to_device(v[None], spec), out)
+        if t % 8 and t not in att:
+            continue
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        tag = f"{spec.name} window {t}"
+        n = res["n"]
+        if n:
+            pu.assert_rel(pu.to_numpy(st.scores[0, :, :n]), res["scores"], 1.0, tag + " scores")
+        nd = pu.compare_selection(pu.to_numpy(st.sel_idx[0]).astype(np.int64), int(st.sel_count.item()), res, tag)
+        assert nd >= 0
+        near += nd
+        if t in att and nd == 0:
+            pu.assert_attention(pu.to_numpy(out), res["out"], tag + " attention")
+    sel = pu.to_numpy(st.sel_idx[0]).astype(int)
+    for g in range(spec.n_kv_heads):
+        assert set(wl.planted_blocks(spec, 0)[g]) <= set(sel[g])
+    print("131k sweep: near-tie differences", near)
+
+
+def test_decode_batch_fixed_probes(B):
+    """Batched decode (Eq. 3): sequences of different lengths, one token per step, 512 recent
+    tokens kept local, probes fixed from each sequence's last prefill window, two layers with
+    the budget chain between them.  Reduced sizes of the 16-sequence workload."""
+    import torch
+    base = wl.decode_batch16()
+    spec = base.replace(n_layers=2, n_seq=3, decode_steps=6, ctx_lo=2048, ctx_hi=6144, context=8192,
+                        k_blocks=8, cap_blocks=16, n_planted=0)
+    L, S = spec.n_layers, spec.n_seq
+    ctx = (wl.decode_contexts(spec) // spec.window) * spec.window          # whole prefill windows
+    cfg = B.make_config(spec, out_dtype=B.F32, max_context=int(ctx.max()) + spec.decode_steps + spec.window,
+                        n_phys_pages=S * (-(-(int(ctx.max()) + spec.decode_steps + 16) // 16)))
+    # one pool of pages per layer shared by the sequences, disjoint seeded page tables
+    per_seq = cfg.n_phys_pages // S
+    rng = np.random.default_rng(5)
+    perm = rng.permutation(cfg.n_phys_pages).astype(np.int32)
+    table = np.zeros((S, cfg.max_pages), np.int32)
+    for s in range(S):
+        table[s, :per_seq] = perm[s * per_seq:(s + 1) * per_seq][: cfg.max_pages][:per_seq]
+    st = B.RetrievalState(cfg, n_seq=S, n_layers=L, page_table=table)
+    # prefill (n_local_prev = 0 during prefill, as in the paper's prefill stage) sequence by sequence
+    # through per-sequence states that alias the shared buffers
+    pre_spec = spec.replace(n_local_prev=0)
+    pre_cfg = B.make_config(pre_spec, out_dtype=B.F32, max_context=cfg.max_pages * 16, n_phys_pages=cfg.n_phys_pages)
+    pre_cfg.n_cap, pre_cfg.max_pages = cfg.n_cap, cfg.max_pages
+    chains = [orc.BudgetChain(L, spec.k_blocks, spec.cap_blocks, "streaming") for _ in range(S)]
+    runners = [[pu.OracleRunner(pre_spec, layer=l, chain=chains[s]) for l in range(L)] for s in range(S)]
+    out_w = torch.zeros(L, spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    probes = np.zeros((S, L, spec.n_kv_heads, spec.head_dim))
+    for s in range(S):
+        ps = B.RetrievalState(pre_cfg, n_seq=1, n_layers=L, page_table=table[s:s + 1], shared_pages=(st.k_pages, st.v_pages))
+        sspec = pre_spec.replace(seed=spec.seed + 100 * s)
+        for t in range(int(ctx[s]) // spec.window):
+            qs, ks, vs = [], [], []
+            for l in range(L):
+                q = wl.gen_q(sspec, l, t); k, v = wl.gen_kv(sspec, l, t)
+                qs.append(q); ks.append(k); vs.append(v)
+                r = runners[s][l].step(q, k, v, attention=False)
+                probes[s, l] = r["probe_kv"]
+            ps.step(pu.to_device(np.stack(qs), spec), pu.to_device(np.stack(ks), spec),
+                    pu.to_device(np.stack(vs), spec), out_w)
+        torch.cuda.synchronize()
+        assert int(ps.status.item()) == 0
+        # hand the sequence's state over to the batched decode state (unit = s * L + l)
+        for name in ("repr_k", "repr_inv_norm", "probe_kv", "probe_qh", "stats_mean", "stats_m2", "stats_count"):
+            getattr(st, name)[s * L:(s + 1) * L].copy_(getattr(ps, name))
+        st.budget_state[s].copy_(ps.budget_state[0])
+        assert np.allclose(pu.to_numpy(ps.probe_kv), probes[s], rtol=1e-3, atol=1e-4)
+    st.set_positions([int(c) for c in ctx])
+    # ---- decode: one token per sequence per step, probes fixed
+    for l in range(L):
+        for s in range(S):
+            runners[s][l].spec = spec                      # 512 local tokens from here on
+    out = torch.zeros(S * L, 1, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    rs = np.random.default_rng(9)
+    for step in range(spec.decode_steps):
+        q = wl.bf16_grid(rs.standard_normal((S * L, 1, spec.n_q_heads, spec.head_dim)).astype(np.float32))
+        k = wl.bf16_grid(rs.standard_normal((S * L, 1, spec.n_kv_heads, spec.head_dim)).astype(np.float32))
+        v = wl.bf16_grid(rs.standard_normal((S * L, 1, spec.n_kv_heads, spec.head_dim)).astype(np.float32))
+        st.step(pu.to_device(q, spec), pu.to_device(k, spec), pu.to_device(v, spec), out, n_tokens=1,
+                update_probe=False)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        for s in range(S):
+            for l in range(L):
+                u = s * L + l
+                run = runners[s][l]
+                state = run.state
+                p0 = state.k_cache.shape[0]
+                n = orc.n_candidate_blocks(p0, spec.n_init, spec.block, spec.n_local_prev)
+                run._extend_table(run.complete_blocks())
+                sc = orc.block_scores(probes[s, l], run.table[:, :n])
+                theta = orc.information_density(sc)
+                c, b_real, fragile = chains[s].grant(l, theta, n)
+                sel = [orc.select_blocks(sc[g], c)[0] for g in range(spec.n_kv_heads)]
+                o, _ = orc.retrieval_attention(q[u], k[u], v[u], state.k_cache, state.v_cache, p0, sel, spec.n_init,
+                                               spec.block, spec.n_local_prev)
+                state.k_cache, state.v_cache = orc.append_window(state.k_cache, state.v_cache, k[u], v[u])
+                tag = f"decode step {step} seq {s} layer {l}"
+                if fragile:
+                    continue
+                assert int(st.sel_count[u].item()) == c, tag
+                got = pu.to_numpy(st.sel_idx[u]).astype(np.int64)
+                for g in range(spec.n_kv_heads):
+                    _, tau, near = orc.select_blocks(sc[g], c)
+                    diff = set(got[g][:c].tolist()) ^ set(sel[g].tolist())
+                    assert diff <= set(near.tolist()), tag
+                    if diff:
+                        break
+                else:
+                    pu.assert_attention(pu.to_numpy(out[u]), o, tag + " attention")
