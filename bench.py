@@ -128,6 +128,23 @@ def stage_bytes(spec, p0):
     }
 
 
+def max_over_ranks(x: float, device=None) -> float:
+    """The slowest rank's value (all ranks get it); the identity when there is one process."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Whole-job units per second: every rank processes its own units (independent layers, no
+    collective on the data path), the step time is the slowest rank's."""
+    return world * units_per_rank_step / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------
 def build_states(spec, n_copies, device):
     """Prefills one layer up to the last window on the GPU, then clones the state into
@@ -231,13 +248,9 @@ def run_ours(args):
     sampler.sample()
     barrier()
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), device)
     ms_step = ms_total / args.steps
-    value = world * spec.window / (ms_step * 1e-3)
+    value = job_throughput(spec.window, world, ms_step)
 
     # instrumented pass: per-stage device time with events around each call
     events = {}
@@ -281,11 +294,7 @@ def run_ours(args):
     t0 = time.perf_counter()
     for i in range(e2e_steps):
         e2e_step(3 + i)
-    t_e2e = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([t_e2e], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_e2e = float(t.item())
+    t_e2e = max_over_ranks(time.perf_counter() - t0, device)
     e2e = {"value": world * spec.window * e2e_steps / t_e2e, "unit": UNIT,
            "h2d_bytes_per_step": int(hq.numel() + hk.numel() + hv.numel()) * 2,
            "d2h_bytes_per_step": int(ho.numel()) * 2, "steps": e2e_steps}
