@@ -199,13 +199,40 @@ int actqkv_score_select(const actqkv_config* cfg, const actqkv_batch* batch, con
  *   sel_idx, sel_count                  as written by select_cutoff
  *   out          [U][n_tokens][Hq][D]   cfg->out_dtype out
  *   lse          [U][Hq][n_tokens]      fp32 out, may be NULL (natural-log sum of exp)
- * bf16, D = 128, B = 128, n_tokens and p0 multiples of 128 run on the tcgen05 tensor-core
- * kernel; every other shape runs on the general fp32-accumulate kernel. */
+ * bf16, D = 128, 16-token pages: steps whose n_tokens is a multiple of 128 run on the tcgen05
+ * prefill kernels (CTA pairs when G is even), steps of n_tokens <= 128 / G tokens on the tcgen05
+ * decode kernel (one CTA per KV head; see actqkv_decode_attention for the split form); every
+ * other shape runs on the general fp32-accumulate kernel. */
 int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
                                const void* k_win, const void* v_win, int32_t n_tokens,
                                const void* k_pages, const void* v_pages, const int32_t* page_table,
                                const int64_t* pos0, const int32_t* sel_idx, const int32_t* sel_count,
                                void* out, float* lse, int32_t* status, void* stream);
+
+/* ---- step 5 for short steps (decode, Eq. 3) with the key stream split over several CTAs --------
+ * The same attention as actqkv_retrieval_attention for steps of n_tokens <= 128 / G tokens
+ * (G = Hq / Hkv; bf16, D = 128, 16-token pages), which packs the G query heads of a KV head into
+ * one tensor-core tile so that K and V are read once per group.  With few (sequence, layer) units a
+ * single CTA per KV head cannot fill the GPU: n_splits > 1 cuts every key stream into n_splits
+ * shares; each share writes a partial result to `workspace` and a second kernel merges them
+ * (n_splits = 0 picks the count that fills the SMs once; actqkv_decode_splits returns it).
+ *   workspace  device scratch of at least actqkv_decode_workspace_bytes(...) bytes, 16-byte
+ *              aligned, caller-owned, contents undefined on entry and exit; may be NULL when
+ *              the split count is 1.  Calls that overlap on the GPU need distinct workspaces.
+ * The rows of the last, partly filled cache page that lie past p0 must hold finite values
+ * (e.g. a zero-initialised pool): they are masked out of the softmax but still enter the
+ * P V product with weight 0.
+ * Returns ACTQKV_ERR_UNSUPPORTED for shapes this kernel does not serve, ACTQKV_ERR_SHAPE when
+ * workspace_bytes is too small. */
+int32_t actqkv_decode_splits(const actqkv_config* cfg, const actqkv_batch* batch);
+int64_t actqkv_decode_workspace_bytes(const actqkv_config* cfg, const actqkv_batch* batch, int32_t n_tokens,
+                                      int32_t n_splits);
+int actqkv_decode_attention(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
+                            const void* k_win, const void* v_win, int32_t n_tokens, const void* k_pages,
+                            const void* v_pages, const int32_t* page_table, const int64_t* pos0,
+                            const int32_t* sel_idx, const int32_t* sel_count, void* out, float* lse,
+                            int32_t n_splits, void* workspace, int64_t workspace_bytes, int32_t* status,
+                            void* stream);
 
 /* ---- step 6: cache append (Eq. 4) and representatives of the completed blocks ----------
  * Copies the step's keys / values into the pages of tokens [p0, p0 + n_tokens) and, for every

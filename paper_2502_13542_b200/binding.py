@@ -75,6 +75,9 @@ _SIGS = {
     "actqkv_score_select": ([_P] * 14, C.c_int),
     "actqkv_retrieval_attention": ([_P, _P, _P, _P, _P, C.c_int32] + [_P] * 10, C.c_int),
     "actqkv_append_window": ([_P, _P, _P, _P, C.c_int32] + [_P] * 8, C.c_int),
+    "actqkv_decode_splits": ([_P, _P], C.c_int32),
+    "actqkv_decode_workspace_bytes": ([_P, _P, C.c_int32, C.c_int32], C.c_int64),
+    "actqkv_decode_attention": ([_P, _P, _P, _P, _P, C.c_int32] + [_P] * 8 + [C.c_int32, _P, C.c_int64, _P, _P], C.c_int),
 }
 for _name, (_args, _res) in _SIGS.items():
     _fn = getattr(_lib, _name)          # AttributeError if the library lacks a declared symbol
@@ -166,6 +169,23 @@ def retrieval_attention(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages,
                                            n_tokens, _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
                                            _ptr(pos0), _ptr(sel_idx), _ptr(sel_count), _ptr(out),
                                            _ptr(lse), _ptr(status), _stream()))
+
+
+def decode_splits(cfg, batch) -> int:
+    return _lib.actqkv_decode_splits(C.byref(cfg), _b(batch))
+
+
+def decode_workspace_bytes(cfg, batch, n_tokens, n_splits=0) -> int:
+    return _lib.actqkv_decode_workspace_bytes(C.byref(cfg), _b(batch), n_tokens, n_splits)
+
+
+def decode_attention(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages, page_table, pos0,
+                     sel_idx, sel_count, out, lse=None, n_splits=0, workspace=None, status=None):
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(_lib.actqkv_decode_attention(C.byref(cfg), _b(batch), _ptr(q), _ptr(k_win), _ptr(v_win), n_tokens,
+                                        _ptr(k_pages), _ptr(v_pages), _ptr(page_table), _ptr(pos0),
+                                        _ptr(sel_idx), _ptr(sel_count), _ptr(out), _ptr(lse), n_splits,
+                                        _ptr(workspace), ws_bytes, _ptr(status), _stream()))
 
 
 def append_window(cfg, batch, k_win, v_win, n_tokens, pos0, k_pages, v_pages, page_table, repr_k,

@@ -61,5 +61,52 @@ extern "C" int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv
   const bool tc1_only = force && std::strcmp(force, "tc1") == 0;
   if (!simt_only && !tc1_only && attention_tc2_supported(cfg, n_tokens)) return launch_attention_tc2(cfg, b, a, st);
   if (!simt_only && attention_tc_supported(cfg, n_tokens)) return launch_attention_tc(cfg, b, a, st);
+  if (!simt_only && attention_decode_supported(cfg, n_tokens)) return launch_attention_decode(cfg, b, a, 1, nullptr, st);
   return launch_attention_simt(cfg, b, a, st);
+}
+
+extern "C" int32_t actqkv_decode_splits(const actqkv_config* cfg, const actqkv_batch* batch) {
+  const Batch b = get_batch(batch);
+  if (check_config(cfg, b)) return 0;
+  return attention_decode_auto_splits(cfg, b);
+}
+
+extern "C" int64_t actqkv_decode_workspace_bytes(const actqkv_config* cfg, const actqkv_batch* batch, int32_t n_tokens,
+                                                 int32_t n_splits) {
+  const Batch b = get_batch(batch);
+  if (check_config(cfg, b) || n_tokens <= 0) return 0;
+  if (n_splits <= 0) n_splits = attention_decode_auto_splits(cfg, b);
+  return attention_decode_workspace_bytes(cfg, b, n_tokens, n_splits);
+}
+
+extern "C" int actqkv_decode_attention(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
+                                       const void* k_win, const void* v_win, int32_t n_tokens, const void* k_pages,
+                                       const void* v_pages, const int32_t* page_table, const int64_t* pos0,
+                                       const int32_t* sel_idx, const int32_t* sel_count, void* out, float* lse,
+                                       int32_t n_splits, void* workspace, int64_t workspace_bytes, int32_t* status,
+                                       void* stream) {
+  const Batch b = get_batch(batch);
+  int rc = check_config(cfg, b);
+  if (rc) return rc;
+  ACTQKV_REQUIRE_PTR(q);
+  ACTQKV_REQUIRE_PTR(k_win);
+  ACTQKV_REQUIRE_PTR(v_win);
+  ACTQKV_REQUIRE_PTR(k_pages);
+  ACTQKV_REQUIRE_PTR(v_pages);
+  ACTQKV_REQUIRE_PTR(out);
+  ACTQKV_OPTIONAL_PTR(lse);
+  ACTQKV_OPTIONAL_PTR(workspace);
+  if (!page_table || !pos0) return ACTQKV_ERR_NULL;
+  if (cfg->cap_blocks > 0 && (!sel_idx || !sel_count)) return ACTQKV_ERR_NULL;
+  if (n_tokens <= 0 || n_tokens > cfg->window) return ACTQKV_ERR_SHAPE;
+  if (!attention_decode_supported(cfg, n_tokens)) return ACTQKV_ERR_UNSUPPORTED;
+  if (n_splits <= 0) n_splits = attention_decode_auto_splits(cfg, b);
+  if (n_splits > 64) return ACTQKV_ERR_SHAPE;
+  const int64_t need = attention_decode_workspace_bytes(cfg, b, n_tokens, n_splits);
+  if (need > 0 && (!workspace || workspace_bytes < need)) return workspace ? ACTQKV_ERR_SHAPE : ACTQKV_ERR_NULL;
+  AttnArgs a;
+  a.q = q; a.k_win = k_win; a.v_win = v_win; a.k_pages = k_pages; a.v_pages = v_pages;
+  a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
+  a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
+  return launch_attention_decode(cfg, b, a, n_splits, workspace, reinterpret_cast<cudaStream_t>(stream));
 }

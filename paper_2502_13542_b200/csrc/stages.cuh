@@ -46,4 +46,12 @@ int launch_attention_tc(const actqkv_config* cfg, const Batch& b, const AttnArgs
 bool attention_tc2_supported(const actqkv_config* cfg, int n_tokens);
 int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 
+// Short steps (decode): one CTA per (unit, KV head, split of the key stream), G query heads packed
+// in the M tile; n_splits > 1 needs a workspace of attention_decode_workspace_bytes().
+bool attention_decode_supported(const actqkv_config* cfg, int n_tokens);
+int attention_decode_auto_splits(const actqkv_config* cfg, const Batch& b);
+int64_t attention_decode_workspace_bytes(const actqkv_config* cfg, const Batch& b, int n_tokens, int n_splits);
+int launch_attention_decode(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, int n_splits,
+                            void* workspace, cudaStream_t st);
+
 }  // namespace actqkv

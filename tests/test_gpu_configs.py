@@ -214,3 +214,55 @@ def test_decode_batch_fixed_probes(B):
                         break
                 else:
                     pu.assert_attention(pu.to_numpy(out[u]), o, tag + " attention")
+
+
+@pytest.mark.parametrize("n_new", [1, 5, 32])
+def test_decode_attention_splits_match_general_kernel(B, monkeypatch, n_new):
+    """The tensor-core decode kernel, unsplit and with the key stream cut into 2, 5, 16 and the
+    automatic number of shares (workspace + merge kernel), against the general fp32 kernel on the
+    same state: ragged position (the last cache page partly filled), 512 local tokens, steps of
+    1, 5 and 32 = 128 / G new tokens."""
+    import torch
+    spec = wl.llama3_8b_layer().replace(context=4096, n_local_prev=512, k_blocks=16, cap_blocks=16)
+    cfg = B.make_config(spec, out_dtype=B.F32, max_context=8192)
+    st = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, 8192)[None, :])
+    out_w = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    for t in range(spec.n_windows):
+        q = pu.to_device(wl.gen_q(spec, 0, t)[None], spec)
+        k, v = wl.gen_kv(spec, 0, t)
+        st.step(q, pu.to_device(k[None], spec), pu.to_device(v[None], spec), out_w)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    def rnd(n, h):
+        return torch.randn(1, n, h, spec.head_dim, device="cuda", generator=g).to(torch.bfloat16)
+    o1 = torch.zeros(1, 1, spec.n_q_heads, spec.head_dim, device="cuda")
+    for _ in range(19):                                   # leaves p0 = 4096 + 19: not on a page boundary
+        st.step(rnd(1, spec.n_q_heads), rnd(1, spec.n_kv_heads), rnd(1, spec.n_kv_heads), o1, n_tokens=1,
+                update_probe=False)
+    q, k, v = rnd(n_new, spec.n_q_heads), rnd(n_new, spec.n_kv_heads), rnd(n_new, spec.n_kv_heads)
+    B.score_select(cfg, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, st.budget_state, st.scores,
+                   st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
+    shape = (1, n_new, spec.n_q_heads, spec.head_dim)
+    ref, ref_lse = torch.zeros(shape, device="cuda"), torch.zeros(spec.n_q_heads, n_new, device="cuda")
+    monkeypatch.setenv("ACTQKV_ATTENTION", "simt")
+    B.retrieval_attention(cfg, st.batch, q, k, v, n_new, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                          st.sel_count, ref, ref_lse, st.status)
+    torch.cuda.synchronize()
+    monkeypatch.delenv("ACTQKV_ATTENTION")
+    auto = B.decode_splits(cfg, st.batch)
+    assert auto >= 8                                      # 8 (unit, KV head) pairs on a GPU of ~148 SMs
+    for splits in (1, 2, 5, 16, 0):
+        ws_bytes = B.decode_workspace_bytes(cfg, st.batch, n_new, splits)
+        assert (ws_bytes == 0) == (splits == 1)
+        ws = torch.full((max(ws_bytes, 16) // 4,), float("nan"), device="cuda")
+        got, lse = torch.full(shape, float("nan"), device="cuda"), torch.zeros_like(ref_lse)
+        B.decode_attention(cfg, st.batch, q, k, v, n_new, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                           st.sel_count, got, lse, n_splits=splits, workspace=ws if splits != 1 else None,
+                           status=st.status)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        assert (got - ref).abs().max().item() < 4e-3, splits
+        assert (lse - ref_lse).abs().max().item() < 2e-3, splits
+    # a workspace that is too small is refused on the host
+    with pytest.raises(B.ActQKVError):
+        B.decode_attention(cfg, st.batch, q, k, v, n_new, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                           st.sel_count, got, lse, n_splits=4, workspace=torch.zeros(64, device="cuda"))
