@@ -59,7 +59,8 @@ typedef enum actqkv_status {
   ACTQKV_ERR_SHAPE = -3,        /* unsupported head_dim / window / block ...  */
   ACTQKV_ERR_DTYPE = -4,        /* dtype not supported by this entry point    */
   ACTQKV_ERR_LAUNCH = -5,       /* the CUDA runtime refused the launch        */
-  ACTQKV_ERR_UNSUPPORTED = -6   /* valid request this build cannot serve      */
+  ACTQKV_ERR_UNSUPPORTED = -6,  /* valid request this build cannot serve      */
+  ACTQKV_ERR_SCRATCH_LIMIT = -7 /* needs more than the built-in scratch array */
 } actqkv_status;
 
 /* bits ORed into *status by kernels */
@@ -233,6 +234,34 @@ int actqkv_decode_attention(const actqkv_config* cfg, const actqkv_batch* batch,
                             const int32_t* sel_idx, const int32_t* sel_count, void* out, float* lse,
                             int32_t n_splits, void* workspace, int64_t workspace_bytes, int32_t* status,
                             void* stream);
+
+/* ---- the split decode attention for callers that cannot allocate device memory ---------------
+ * (An addition of this library; the paper has no counterpart.)
+ * actqkv_decode_attention needs a caller-allocated workspace as soon as the key stream is split.
+ * Some callers cannot provide one: an inference server that hands all of the GPU's memory to its
+ * KV-cache pool at start-up and forbids allocations afterwards, or a per-token decode loop in
+ * which a cudaMalloc (which synchronises the whole device) is not acceptable.  For them this
+ * variant computes exactly the same result with the scratch taken from a fixed array of
+ * ACTQKV_STATIC_SCRATCH_BYTES (8 MiB) that is part of the library's device image.  It calls no
+ * allocation routine of any kind.
+ *  - The array exists once per GPU that loads the library and stays reserved until the process
+ *    ends, used or not.
+ *  - A call whose scratch need (actqkv_decode_workspace_bytes for the same arguments) exceeds
+ *    the array returns ACTQKV_ERR_SCRATCH_LIMIT and enqueues nothing: use fewer splits, or the
+ *    workspace form.
+ *  - The first call on each device looks up that device's copy of the array (the device must be
+ *    current, as for every call).  Make that first call before any stream capture begins.
+ *  - All calls on a device share the one array and it keeps whatever the last call wrote.  The
+ *    kernels never read stale contents, so nothing has to be cleared, but two calls that may
+ *    run at the same time on one GPU (different streams) race on it: serialise them, or give
+ *    all but one of them the workspace form.
+ * Arguments and results as actqkv_decode_attention, without workspace and workspace_bytes. */
+#define ACTQKV_STATIC_SCRATCH_BYTES (8u << 20)
+int actqkv_decode_attention_static(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
+                                   const void* k_win, const void* v_win, int32_t n_tokens, const void* k_pages,
+                                   const void* v_pages, const int32_t* page_table, const int64_t* pos0,
+                                   const int32_t* sel_idx, const int32_t* sel_count, void* out, float* lse,
+                                   int32_t n_splits, int32_t* status, void* stream);
 
 /* ---- step 6: cache append (Eq. 4) and representatives of the completed blocks ----------
  * Copies the step's keys / values into the pages of tokens [p0, p0 + n_tokens) and, for every

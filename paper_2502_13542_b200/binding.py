@@ -77,6 +77,7 @@ _SIGS = {
     "actqkv_append_window": ([_P, _P, _P, _P, C.c_int32] + [_P] * 8, C.c_int),
     "actqkv_decode_splits": ([_P, _P], C.c_int32),
     "actqkv_decode_workspace_bytes": ([_P, _P, C.c_int32, C.c_int32], C.c_int64),
+    "actqkv_decode_attention_static": ([_P, _P, _P, _P, _P, C.c_int32] + [_P] * 8 + [C.c_int32, _P, _P], C.c_int),
     "actqkv_decode_attention": ([_P, _P, _P, _P, _P, C.c_int32] + [_P] * 8 + [C.c_int32, _P, C.c_int64, _P, _P], C.c_int),
 }
 for _name, (_args, _res) in _SIGS.items():
@@ -186,6 +187,19 @@ def decode_attention(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages, pa
                                         _ptr(k_pages), _ptr(v_pages), _ptr(page_table), _ptr(pos0),
                                         _ptr(sel_idx), _ptr(sel_count), _ptr(out), _ptr(lse), n_splits,
                                         _ptr(workspace), ws_bytes, _ptr(status), _stream()))
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def decode_attention_static(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages, page_table, pos0,
+                            sel_idx, sel_count, out, lse=None, n_splits=0, status=None):
+    """The split decode attention with the library's own fixed scratch array: no workspace
+    argument and no allocation.  Calls that may overlap on one GPU must not both use it."""
+    _check(_lib.actqkv_decode_attention_static(C.byref(cfg), _b(batch), _ptr(q), _ptr(k_win), _ptr(v_win),
+                                               n_tokens, _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
+                                               _ptr(pos0), _ptr(sel_idx), _ptr(sel_count), _ptr(out), _ptr(lse),
+                                               n_splits, _ptr(status), _stream()))
 
 
 def append_window(cfg, batch, k_win, v_win, n_tokens, pos0, k_pages, v_pages, page_table, repr_k,

@@ -18,6 +18,7 @@ extern "C" const char* actqkv_strerror(int status) {
     case ACTQKV_ERR_DTYPE: return "unsupported dtype";
     case ACTQKV_ERR_LAUNCH: return "the CUDA runtime refused the launch";
     case ACTQKV_ERR_UNSUPPORTED: return "valid request this build cannot serve";
+    case ACTQKV_ERR_SCRATCH_LIMIT: return "the call needs more scratch than the library's built-in array holds";
     default: return "unknown actqkv status";
   }
 }

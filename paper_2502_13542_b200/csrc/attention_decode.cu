@@ -531,3 +531,70 @@ int launch_attention_decode(const actqkv_config* cfg, const Batch& b, const Attn
 }
 
 }  // namespace actqkv
+
+// ---------------------------------------------------------------- entry point that allocates nothing
+namespace {
+
+// Scratch for the split form of the decode attention, owned by the library image itself: the
+// array is part of the module, so every device that loads the library reserves these bytes from
+// load until the process exits, and no allocation call is ever needed to use them.
+static __device__ __align__(256) unsigned char g_decode_scratch[ACTQKV_STATIC_SCRATCH_BYTES];
+
+// In host code `g_decode_scratch` is only a handle for the runtime, not a device address; the
+// address of each device's copy is asked for once, with that device current, and remembered.
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {};
+
+int static_scratch(void** ptr) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ACTQKV_ERR_LAUNCH;
+  if (!g_scratch_addr[dev]) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_decode_scratch) != cudaSuccess || !addr) {
+      (void)cudaGetLastError();
+      return ACTQKV_ERR_LAUNCH;
+    }
+    g_scratch_addr[dev] = addr;
+  }
+  *ptr = g_scratch_addr[dev];
+  return ACTQKV_OK;
+}
+
+}  // namespace
+
+extern "C" int actqkv_decode_attention_static(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
+                                              const void* k_win, const void* v_win, int32_t n_tokens,
+                                              const void* k_pages, const void* v_pages, const int32_t* page_table,
+                                              const int64_t* pos0, const int32_t* sel_idx, const int32_t* sel_count,
+                                              void* out, float* lse, int32_t n_splits, int32_t* status, void* stream) {
+  const Batch b = get_batch(batch);
+  int rc = check_config(cfg, b);
+  if (rc) return rc;
+  ACTQKV_REQUIRE_PTR(q);
+  ACTQKV_REQUIRE_PTR(k_win);
+  ACTQKV_REQUIRE_PTR(v_win);
+  ACTQKV_REQUIRE_PTR(k_pages);
+  ACTQKV_REQUIRE_PTR(v_pages);
+  ACTQKV_REQUIRE_PTR(out);
+  ACTQKV_OPTIONAL_PTR(lse);
+  if (!page_table || !pos0) return ACTQKV_ERR_NULL;
+  if (cfg->cap_blocks > 0 && (!sel_idx || !sel_count)) return ACTQKV_ERR_NULL;
+  if (n_tokens <= 0 || n_tokens > cfg->window) return ACTQKV_ERR_SHAPE;
+  if (!attention_decode_supported(cfg, n_tokens)) return ACTQKV_ERR_UNSUPPORTED;
+  if (n_splits <= 0) n_splits = attention_decode_auto_splits(cfg, b);
+  if (n_splits > 64) return ACTQKV_ERR_SHAPE;
+  if (attention_decode_workspace_bytes(cfg, b, n_tokens, n_splits) > int64_t(ACTQKV_STATIC_SCRATCH_BYTES))
+    return ACTQKV_ERR_SCRATCH_LIMIT;
+  void* scratch = nullptr;
+  rc = static_scratch(&scratch);
+  if (rc) return rc;
+  AttnArgs a;
+  a.q = q; a.k_win = k_win; a.v_win = v_win; a.k_pages = k_pages; a.v_pages = v_pages;
+  a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
+  a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
+  // Nothing in the scratch has to start at zero: every split writes its log-sum-exp (minus
+  // infinity when it holds no tile) and the merge reads a partial output only where that value
+  // is finite, so what an earlier call left behind is never read.
+  return launch_attention_decode(cfg, b, a, n_splits, scratch, reinterpret_cast<cudaStream_t>(stream));
+}
+
