@@ -406,6 +406,164 @@ def run_reference(args):
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
+# ------------------------------------------------------------------------------------------
+# Secondary workloads (not the default headline line): the memory-bound stages on batched shapes
+def _device_activations(spec, shape_heads, device, gen, n_tokens):
+    """Seeded N(0,1) activations with the workload's outlier channels, drawn on the device
+    (bench-only inputs: the parity tests use the host generator of workloads.py)."""
+    import torch
+    x = torch.randn(*shape_heads[:-1], n_tokens, shape_heads[-1], spec.head_dim, device=device, generator=gen)
+    x[..., : spec.n_outlier] *= spec.outlier_scale
+    return x.to(torch.bfloat16)
+
+
+def _time_stage(fn, iters, flush):
+    import torch
+    evs = []
+    for _ in range(iters):
+        flush()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    t = sorted(a.elapsed_time(b) for a, b in evs)
+    return 1e3 * t[len(t) // 2]          # median, microseconds
+
+
+def run_stack32(args):
+    """All 32 layers of the LLaMA3-8B shape batched in one launch per stage at the last window of a
+    32k prefill: Q = 134 MB, representative table = 66 MB per launch (larger than or comparable
+    to L2; L2 is flushed before every timed launch)."""
+    import torch
+    from paper_2502_13542_b200 import binding as B
+    from paper_2502_13542_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    spec = wl.llama3_8b_stack32()
+    L = spec.n_layers
+    cfg = B.make_config(spec, out_dtype=B.BF16)
+    st = B.RetrievalState(cfg, n_seq=1, n_layers=L, page_table=wl.shuffled_page_table(spec, spec.context)[None, :], device=dev)
+    gen = torch.Generator(device=dev).manual_seed(spec.seed)
+    out = torch.zeros(L, spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=dev)
+    W = spec.window
+    for t in range(spec.n_windows - 1):
+        q = _device_activations(spec, (L, spec.n_q_heads), dev, gen, W)
+        k = _device_activations(spec, (L, spec.n_kv_heads), dev, gen, W)
+        v = _device_activations(spec, (L, spec.n_kv_heads), dev, gen, W)
+        st.step(q, k, v, out)
+    q = _device_activations(spec, (L, spec.n_q_heads), dev, gen, W)
+    k = _device_activations(spec, (L, spec.n_kv_heads), dev, gen, W)
+    v = _device_activations(spec, (L, spec.n_kv_heads), dev, gen, W)
+    torch.cuda.synchronize()
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flush = lambda: scratch.fill_(1)
+    b = st.batch
+    p0 = (spec.n_windows - 1) * W
+    sb = stage_bytes(spec, p0)
+    stages = {
+        "bias_probe": (lambda: B.bias_probe(cfg, b, q, W, st.stats_count, st.stats_mean, st.stats_m2, st.phi_l1, None,
+                                            st.probe_qh, st.probe_kv, st.status), L * sb["bias_probe"]),
+        "score_select": (lambda: B.score_select(cfg, b, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand,
+                                                st.budget_state, st.scores, st.theta, st.sel_idx, st.sel_count,
+                                                st.budget_real, st.status), L * (sb["score"] + sb["select"])),
+        "append": (lambda: B.append_window(cfg, b, k, v, W, st.pos0, st.k_pages, st.v_pages, st.page_table,
+                                           st.repr_k, st.repr_inv_norm, st.status), L * sb["append"]),
+    }
+    peaks = load_peaks()
+    res = {}
+    for name, (fn, nbytes) in stages.items():
+        for _ in range(3):
+            fn()
+        us = _time_stage(fn, args.steps if args.steps < 100 else 30, flush)
+        res[name] = {"us": us, "bytes": nbytes, "GBps": nbytes / us / 1e3, "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+    assert int(st.status.item()) == 0
+    print(json.dumps({"workload": "llama3_8b_stack32_32k: 32 layers batched per launch, last window", "stages": res,
+                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cold_l2": "512 MB fill before every timed launch"}))
+
+
+def run_decode16(args):
+    """Decode, 16 sequences with contexts ~ U[32768, 131072], one token per step, one layer per
+    launch, probes fixed: score + cut-off/select over every sequence's table, then the decode
+    attention over [128 initial | 32 selected blocks | >= 512 local] keys per KV head."""
+    import torch
+    from paper_2502_13542_b200 import binding as B
+    from paper_2502_13542_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    spec = wl.decode_batch16().replace(n_layers=1, cap_blocks=32)
+    S = spec.n_seq
+    ctx = (wl.decode_contexts(spec) // spec.window) * spec.window
+    n_pools = 2                                             # distinct physical layer copies, rotated
+    max_ctx = int(ctx.max()) + spec.window
+    pages_per_seq = -(-max_ctx // 16)
+    cfg = B.make_config(spec, out_dtype=B.BF16, max_context=max_ctx, n_phys_pages=S * pages_per_seq)
+    gen = torch.Generator(device=dev).manual_seed(spec.seed)
+    rng = np.random.default_rng(spec.seed)
+    table = rng.permutation(S * pages_per_seq).astype(np.int32).reshape(S, pages_per_seq)[:, : cfg.max_pages]
+    states = []
+    pre_spec = spec.replace(n_local_prev=0)
+    pre_cfg = B.make_config(pre_spec, out_dtype=B.BF16, max_context=max_ctx, n_phys_pages=S * pages_per_seq)
+    for pool in range(n_pools):
+        st = B.RetrievalState(cfg, n_seq=S, n_layers=1, page_table=table, device=dev)
+        outw = torch.zeros(1, spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=dev)
+        for s_i in range(S):
+            ps = B.RetrievalState(pre_cfg, n_seq=1, n_layers=1, page_table=table[s_i:s_i + 1], device=dev,
+                                  shared_pages=(st.k_pages, st.v_pages))
+            for t in range(int(ctx[s_i]) // spec.window):
+                qw = _device_activations(spec, (1, spec.n_q_heads), dev, gen, spec.window)
+                kw = _device_activations(spec, (1, spec.n_kv_heads), dev, gen, spec.window)
+                vw = _device_activations(spec, (1, spec.n_kv_heads), dev, gen, spec.window)
+                ps.step(qw, kw, vw, outw)
+            for name in ("repr_k", "repr_inv_norm", "probe_kv", "probe_qh"):
+                getattr(st, name)[s_i:s_i + 1].copy_(getattr(ps, name))
+            st.budget_state[s_i].copy_(ps.budget_state[0])
+            del ps
+        st.set_positions([int(c) for c in ctx])
+        states.append(st)
+    torch.cuda.synchronize()
+    q = _device_activations(spec, (S, spec.n_q_heads), dev, gen, 1)
+    k = _device_activations(spec, (S, spec.n_kv_heads), dev, gen, 1)
+    v = _device_activations(spec, (S, spec.n_kv_heads), dev, gen, 1)
+    out = torch.zeros(S, 1, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=dev)
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flush = lambda: scratch.fill_(1)
+    it = {"i": 0}
+
+    def cur():
+        return states[it["i"] % n_pools]
+
+    def score_select():
+        st = cur()
+        B.score_select(cfg, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, st.budget_state, st.scores,
+                       st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
+
+    def attention():
+        st = cur()
+        B.retrieval_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                              st.sel_count, out, None, st.status)
+        it["i"] += 1
+    e = 2
+    n_blocks = [wl.n_candidates(spec, int(c)) for c in ctx]
+    score_bytes = sum(n * spec.n_kv_heads * spec.n_repr * (spec.head_dim * e + 4) + n * spec.n_kv_heads * 4 for n in n_blocks)
+    for st in states:
+        score_select_st = st
+    score_select(); torch.cuda.synchronize()
+    c_sel = cur().sel_count.cpu().numpy()
+    keys = [spec.n_init + int(c_sel[i]) * spec.block + (int(ctx[i]) - (spec.n_init + n_blocks[i] * spec.block)) + 1 for i in range(S)]
+    att_bytes = sum(kk * spec.n_kv_heads * spec.head_dim * e * 2 for kk in keys)
+    peaks = load_peaks()
+    res = {}
+    iters = args.steps if args.steps < 100 else 30
+    for name, fn, nbytes in (("score_select", score_select, score_bytes), ("attention_decode", attention, att_bytes)):
+        for _ in range(3):
+            fn()
+        us = _time_stage(fn, iters, flush)
+        res[name] = {"us": us, "bytes": nbytes, "GBps": nbytes / us / 1e3, "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+    assert all(int(st.status.item()) == 0 for st in states)
+    print(json.dumps({"workload": f"decode16: 16 sequences, contexts {int(ctx.min())}..{int(ctx.max())}, 1 token per step, one layer per launch, {n_pools} layer pools rotated",
+                      "keys_per_head": {"min": min(keys), "max": max(keys)}, "stages": res,
+                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cold_l2": "512 MB fill before every timed launch"}))
+
 
 def main():
     ap = argparse.ArgumentParser()
@@ -416,6 +574,8 @@ def main():
     ap.add_argument("--copies", type=int, default=8)
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="layer32k", choices=["layer32k", "stack32", "decode16"],
+                    help="layer32k = the headline line; the others print per-stage HBM figures on batched shapes")
     ap.add_argument("--profile-region", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
@@ -424,6 +584,10 @@ def main():
         args.steps = min(args.steps, 30)
         args.warmup = min(args.warmup, 2)
         run_reference(args)
+    elif args.workload == "stack32":
+        run_stack32(args)
+    elif args.workload == "decode16":
+        run_decode16(args)
     else:
         run_ours(args)
 
