@@ -48,7 +48,7 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) {
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads) bias_probe_kernel(BiasProbeParams p) {
+__global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams p) {   // 2 CTAs per SM on batched calls
   extern __shared__ __align__(128) unsigned char smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
   constexpr int VN = Vec16<T>::N;             // elements per 16-byte vector

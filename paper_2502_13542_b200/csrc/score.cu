@@ -1,8 +1,8 @@
 // Step 3: cosine scores of the probe-query against every candidate block's representative
 // keys (Eq. 10) and the information density of each head's score distribution (Eq. 11).
 //
-// The representative-key table is streamed once with 16-byte loads.  One warp scores one
-// block: a row of D elements is covered by D*sizeof(T)/16 lanes, all of the warp's loads for
+// The representative-key table is streamed once with 16-byte loads.  One warp scores four
+// blocks: a row of D elements is covered by D*sizeof(T)/16 lanes, all of the warp's loads for
 // the block are issued before the first is used, the dot products are finished with warp
 // shuffles inside each row's lane group.  With one block per warp the grid is wide enough to
 // keep every SM's memory pipeline busy on tables of a few MB.
@@ -14,15 +14,18 @@ using namespace actqkv;
 namespace {
 
 constexpr int kScoreThreads = 256;
-constexpr int kBlocksPerCta = kScoreThreads / 32;   // one candidate block per warp
-constexpr int kMaxPasses = 4;                       // row groups of a block loaded together
+constexpr int kBlocksPerWarp = 4;                   // candidate blocks scored by one warp, loads of all in flight
+constexpr int kBlocksPerCta = (kScoreThreads / 32) * kBlocksPerWarp;
+constexpr int kMaxPasses = 2;                       // row groups of one block held in registers
 
-template <typename T>
+// kMean: block score = mean of the r cosines.  Then every lane scales its partial dot product by
+// its row's inverse norm and ONE shuffle tree over the warp finishes the block; the max
+// aggregation needs the r cosines separately and reduces row by row.
+template <typename T, int D, bool kMean>
 __global__ void __launch_bounds__(kScoreThreads)
 score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
              const float* __restrict__ repr_inv_norm, const int32_t* __restrict__ n_cand,
-             float* __restrict__ scores, int n_kv_heads, int D, int r, int n_cap, int n_layers,
-             int agg_mode, int32_t* status) {
+             float* __restrict__ scores, int n_kv_heads, int r, int n_cap, int n_layers, int32_t* status) {
   const int g = blockIdx.y, unit = blockIdx.z;
   const int seq = unit / n_layers;
   int n = n_cand[seq];
@@ -31,74 +34,103 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
     if (threadIdx.x == 0 && blockIdx.x == 0 && g == 0) set_status(status, ACTQKV_DEV_NCAND_CLAMPED);
   }
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.x * kBlocksPerCta + warp;
-  if (b >= n) return;                     // warp-uniform; no block-wide barrier below
+  const int b0 = (blockIdx.x * (kScoreThreads / 32) + warp) * kBlocksPerWarp;
+  if (b0 >= n) return;                    // warp-uniform; no block-wide barrier below
 
   constexpr int VN = Vec16<T>::N;
-  const int lpr = D / VN;               // lanes per row: 8, 16 or 32
-  const int rows_per_pass = 32 / lpr;
-  const int sub = lane / lpr, lir = lane - sub * lpr;
+  constexpr int LPR = D / VN;           // lanes per row: 8, 16 or 32
+  constexpr int RPP = 32 / LPR;         // rows per pass
+  const int sub = lane / LPR, lir = lane - sub * LPR;
   const size_t head_rows = (size_t(unit) * n_kv_heads + g) * size_t(n_cap) * r;
-  const T* tab = repr_k + (head_rows + size_t(b) * r) * D;
-  const float* inv = repr_inv_norm + head_rows + size_t(b) * r;
+  const int n_pass = (r + RPP - 1) / RPP;
+  const T* tab0 = repr_k + (head_rows + size_t(b0) * r) * D + lir * VN;
+  const float* inv0 = repr_inv_norm + head_rows + size_t(b0) * r;
 
-  // the block's rows first (independent loads), then the probe
-  float kv[kMaxPasses][VN];
-  const int n_pass = (r + rows_per_pass - 1) / rows_per_pass;
+  // every row of the warp's blocks first (independent 16-byte loads), then the probe
+  uint4 kv[kBlocksPerWarp][kMaxPasses];             // raw 16-byte vectors, unpacked at use
+  float nrm[kBlocksPerWarp][kMaxPasses];
 #pragma unroll
-  for (int ps = 0; ps < kMaxPasses; ++ps) {
-    const int i = ps * rows_per_pass + sub;
-    if (ps < n_pass && i < r) Vec16<T>::load_nc(tab + size_t(i) * D + lir * VN, kv[ps]);
-    else {
+  for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
 #pragma unroll
-      for (int e = 0; e < VN; ++e) kv[ps][e] = 0.f;
+    for (int ps = 0; ps < kMaxPasses; ++ps) {
+      const int i = ps * RPP + sub;
+      const bool on = b0 + bi < n && i < r;
+      nrm[bi][ps] = on ? __ldg(inv0 + bi * r + i) : 0.f;
+      kv[bi][ps] = on ? __ldg(reinterpret_cast<const uint4*>(tab0 + (size_t(bi) * r + i) * D)) : make_uint4(0, 0, 0, 0);
     }
   }
-  const float inv_row = lane < r ? __ldg(inv + lane) : 0.f;          // lane i holds 1 / ||R_i||
   const float* pg = probe_kv + (size_t(unit) * n_kv_heads + g) * D;
   float pv[VN];
   Vec16<float>::load_nc(pg + lir * VN, reinterpret_cast<float(&)[4]>(pv[0]));
   if constexpr (VN == 8) Vec16<float>::load_nc(pg + lir * VN + 4, reinterpret_cast<float(&)[4]>(pv[4]));
-  // probe norm: every lane group of lpr lanes holds the whole probe
+  // probe norm: every group of LPR lanes holds the whole probe
   float sq = 0.f;
 #pragma unroll
   for (int e = 0; e < VN; ++e) sq = fmaf(pv[e], pv[e], sq);
-  for (int o = lpr >> 1; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+#pragma unroll
+  for (int o = LPR >> 1; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
   const bool bad = !(sq > 0.f) || !isfinite(sq);
-  if (bad && lane == 0 && b == 0) set_status(status, ACTQKV_DEV_BAD_PROBE);
+  if (bad && lane == 0 && b0 == 0) set_status(status, ACTQKV_DEV_BAD_PROBE);
   const float inv_pn = bad ? 0.f : rsqrtf(sq);
+  float* out = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
 
-  float agg = agg_mode == ACTQKV_AGG_MAX ? -INFINITY : 0.f;
-  for (int p0 = 0; p0 < n_pass; p0 += kMaxPasses) {
-    if (p0 > 0) {                        // more than kMaxPasses row groups: fetch the next batch
 #pragma unroll
-      for (int ps = 0; ps < kMaxPasses; ++ps) {
-        const int i = (p0 + ps) * rows_per_pass + sub;
-        if (p0 + ps < n_pass && i < r) Vec16<T>::load_nc(tab + size_t(i) * D + lir * VN, kv[ps]);
-      }
-    }
+  for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
+    const int b = b0 + bi;
+    if (b >= n) break;                    // warp-uniform
+    if constexpr (kMean) {
+      float acc = 0.f;                    // sum over this lane's rows of (partial dot) / ||R_i||
+      for (int p0 = 0; p0 < n_pass; p0 += kMaxPasses) {
 #pragma unroll
-    for (int ps = 0; ps < kMaxPasses; ++ps) {
-      if (p0 + ps >= n_pass) break;
-      const int i0 = (p0 + ps) * rows_per_pass;
-      float dot = 0.f;
+        for (int ps = 0; ps < kMaxPasses; ++ps) {
+          float row[VN];
+          float w = nrm[bi][ps];
+          if (p0 == 0) {
+            Vec16<T>::unpack(kv[bi][ps], row);
+          } else {                        // more row groups than the registers hold
+            const int i = (p0 + ps) * RPP + sub;
+            w = 0.f;
 #pragma unroll
-      for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], kv[ps][e], dot);
-      for (int o = lpr >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      // combine the row groups of this pass (group leaders hold the dot products)
-      for (int s = 0; s < rows_per_pass; ++s) {
-        const int i = i0 + s;
-        const float d = __shfl_sync(0xffffffffu, dot, s * lpr);
-        const float nrm = i < 32 ? __shfl_sync(0xffffffffu, inv_row, i & 31) : __ldg(inv + min(i, r - 1));
-        if (i < r) {
-          const float cv = d * inv_pn * nrm;
-          agg = agg_mode == ACTQKV_AGG_MAX ? fmaxf(agg, cv) : agg + cv;
+            for (int e = 0; e < VN; ++e) row[e] = 0.f;
+            if (i < r) {
+              w = __ldg(inv0 + bi * r + i);
+              Vec16<T>::load_nc(tab0 + (size_t(bi) * r + i) * D, row);
+            }
+          }
+          float dot = 0.f;
+#pragma unroll
+          for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], row[e], dot);
+          acc = fmaf(dot, w, acc);
         }
       }
+      acc = warp_sum(acc);
+      if (lane == 0) out[b] = acc * inv_pn / float(r);
+    } else {
+      float agg = -INFINITY;
+      for (int ps = 0; ps < n_pass; ++ps) {
+        const int i = ps * RPP + sub;
+        float row[VN];
+        float w = 0.f;
+#pragma unroll
+        for (int e = 0; e < VN; ++e) row[e] = 0.f;
+        if (i < r) {
+          w = __ldg(inv0 + bi * r + i);
+          Vec16<T>::load_nc(tab0 + (size_t(bi) * r + i) * D, row);
+        }
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], row[e], dot);
+#pragma unroll
+        for (int o = LPR >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        float cosv = i < r ? dot * inv_pn * w : -INFINITY;
+        // maximum over the row groups of this pass (group leaders hold the cosines)
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) cosv = fmaxf(cosv, __shfl_xor_sync(0xffffffffu, cosv, o));
+        agg = fmaxf(agg, cosv);
+      }
+      if (lane == 0) out[b] = agg;
     }
   }
-  if (lane == 0)
-    scores[(size_t(unit) * n_kv_heads + g) * n_cap + b] = agg_mode == ACTQKV_AGG_MAX ? agg : agg / float(r);
 }
 
 __global__ void __launch_bounds__(32)
@@ -114,19 +146,33 @@ entropy_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_c
 
 namespace actqkv {
 
+template <typename T, int D>
+void launch_scores_t(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,
+                     const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
+                     cudaStream_t st) {
+  dim3 grid((cfg->n_cap + kBlocksPerCta - 1) / kBlocksPerCta, cfg->n_kv_heads, b.units());
+  if (cfg->agg_mode == ACTQKV_AGG_MAX)
+    score_kernel<T, D, false><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
+                                                              n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
+                                                              cfg->n_cap, b.n_layers, status);
+  else
+    score_kernel<T, D, true><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
+                                                             n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
+                                                             cfg->n_cap, b.n_layers, status);
+}
+
 int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,
                   const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
                   cudaStream_t st) {
   if (cfg->n_cap == 0) return ACTQKV_OK;
-  dim3 grid((cfg->n_cap + kBlocksPerCta - 1) / kBlocksPerCta, cfg->n_kv_heads, b.units());
-  if (cfg->dtype == ACTQKV_BF16)
-    score_kernel<__nv_bfloat16><<<grid, kScoreThreads, 0, st>>>(
-        probe_kv, static_cast<const __nv_bfloat16*>(repr_k), repr_inv_norm, n_cand, scores,
-        cfg->n_kv_heads, cfg->head_dim, cfg->n_repr, cfg->n_cap, b.n_layers, cfg->agg_mode, status);
-  else
-    score_kernel<float><<<grid, kScoreThreads, 0, st>>>(
-        probe_kv, static_cast<const float*>(repr_k), repr_inv_norm, n_cand, scores, cfg->n_kv_heads,
-        cfg->head_dim, cfg->n_repr, cfg->n_cap, b.n_layers, cfg->agg_mode, status);
+  const bool bf16 = cfg->dtype == ACTQKV_BF16;
+  if (cfg->head_dim == 64) {
+    if (bf16) launch_scores_t<__nv_bfloat16, 64>(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
+    else launch_scores_t<float, 64>(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
+  } else {
+    if (bf16) launch_scores_t<__nv_bfloat16, 128>(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
+    else launch_scores_t<float, 128>(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
+  }
   return launch_status();
 }
 

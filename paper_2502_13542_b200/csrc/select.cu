@@ -24,7 +24,7 @@ using namespace actqkv;
 
 namespace {
 
-constexpr int kChainThreads = 256;
+constexpr int kChainThreads = 1024;
 constexpr int kSelThreads = 256;
 
 struct ChainParams {
@@ -80,22 +80,30 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
     for (int g = 0; g < p.n_kv_heads; ++g) s += double(theta_h[l * p.n_kv_heads + g]);
     return s / double(p.n_kv_heads);
   };
+  // Suffix sums over the deeper layers, so that the walk below is linear in L: `known` adds the
+  // theta-bar of the layers that have one (their history mean, or this call's own density in the
+  // Algorithm-1 reading), `open` counts the layers that take the current layer's density instead.
+  // suffix[l] covers layers > l of the MODEL (index = model layer); the batch holds layers
+  // layer0 .. layer0 + Lb - 1.
+  double* suf_known = reinterpret_cast<double*>(theta_h + ((p.Lb * p.n_kv_heads + 1) & ~1));   // [L + 1]
+  double* suf_open = suf_known + p.L + 1;                                                       // [L + 1]
+  suf_known[p.L] = 0.0;
+  suf_open[p.L] = 0.0;
+  for (int j = p.L - 1; j >= 0; --j) {
+    double known = 0.0, open = 0.0;
+    if (p.thetabar_mode == ACTQKV_THETABAR_ALG1) known = layer_theta(j - p.layer0);
+    else if (hist_cnt[j] > 0.0) known = hist_sum[j] / hist_cnt[j];
+    else open = 1.0;
+    suf_known[j] = suf_known[j + 1] + known;
+    suf_open[j] = suf_open[j + 1] + open;
+  }
   for (int l = 0; l < p.Lb; ++l) {
     const int layer = p.layer0 + l;
     if (layer == 0) b_rem = double(p.L) * double(p.k_blocks);
     const double th = layer_theta(l);
     Grant gr{0, 0.0};
     if (n > 0) {
-      double rest = 0.0;
-      for (int j = layer + 1; j < p.L; ++j) {
-        if (p.thetabar_mode == ACTQKV_THETABAR_ALG1) {
-          rest += layer_theta(j - p.layer0);
-        } else if (hist_cnt[j] > 0.0) {
-          rest += hist_sum[j] / hist_cnt[j];
-        } else {
-          rest += th;
-        }
-      }
+      const double rest = suf_known[layer + 1] + suf_open[layer + 1] * th;
       gr = grant_layer(th, rest, b_rem, p.L - layer, n, p.cap_blocks);
       b_rem -= double(gr.c);
       hist_sum[layer] += th;
@@ -324,7 +332,8 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sm_sel)) != cudaSuccess)
     return ACTQKV_ERR_LAUNCH;
   if (!fused) {
-    const size_t sm_chain = sizeof(float) * size_t(b.n_layers) * cfg->n_kv_heads;
+    const size_t sm_chain = sizeof(float) * ((size_t(b.n_layers) * cfg->n_kv_heads + 1) & ~size_t(1)) +
+                            sizeof(double) * 2 * (size_t(cfg->n_layers) + 1);
     if (sm_chain > 48 * 1024) return ACTQKV_ERR_SHAPE;
     cutoff_chain_kernel<<<b.n_seq, kChainThreads, sm_chain, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;
