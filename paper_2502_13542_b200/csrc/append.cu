@@ -171,6 +171,8 @@ extern "C" int actqkv_append_window(const actqkv_config* cfg, const actqkv_batch
   dim3 grid(p.copy_ctas + p.max_new_blocks * cfg->n_kv_heads * cfg->n_repr, b.units());
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const size_t smem = sizeof(double) * size_t(kThreads / vpr) * cfg->head_dim + sizeof(float) * cfg->head_dim;
+  prefer_max_shared(append_kernel<__nv_bfloat16>);
+  prefer_max_shared(append_kernel<float>);
   if (cfg->dtype == ACTQKV_BF16) append_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(p);
   else append_kernel<float><<<grid, kThreads, smem, st>>>(p);
   return launch_status();

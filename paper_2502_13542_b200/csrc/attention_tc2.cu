@@ -9,11 +9,13 @@
 // of M = 256: each CTA supplies its own 128 rows of A (Q from shared memory, P from TMEM) and
 // HALF of B -- 64 of the tile's 128 keys for S = Q K^T, 64 of the 128 channels of V for
 // O += P V -- and receives its own 128 rows of the result in its TMEM.  A CTA therefore loads
-// 32 KiB per tile instead of 64, and the rings hold 6 K halves and 6 V halves.  No TMA multicast
+// 32 KiB per tile instead of 64, and the rings hold 6 K halves and 5 V halves.  No TMA multicast
 // is used: each CTA fetches its own halves.
 //
-// Roles per CTA (384 threads) are those of the single-CTA kernel, except that only the leader
-// CTA (cluster rank 0) issues MMAs.  Cross-CTA signalling:
+// Roles per CTA (640 threads): warp 0 K producer, warp 2 V producer, warps 1 and 3 the MMA issuers
+// (leader CTA = cluster rank 0 only; warp 1: S = Q K^T, warp 3: O += P V), warps 4-19 softmax with
+// FOUR threads per query row (32 key columns each; the four warps of a TMEM lane quadrant share a
+// scheduler, which hides their latencies).  Cross-CTA signalling:
 //   TMA loads of both CTAs complete on the LEADER's "full" barriers (cta_group::2 form of the load);
 //   the leader's commits are multicast to the barriers of both CTAs (slot released, S ready, P V done);
 //   the softmax warps of both CTAs arrive on the leader's "P ready" barrier (one arrival per warp).
@@ -28,18 +30,20 @@ using namespace actqkv::tc;
 namespace {
 
 constexpr int kBM = 128, kBN = 128, kD = 128;
-constexpr int kRing = 6;                                 // K halves in flight, and V halves in flight
+constexpr int kRing = 6;                                 // K halves in flight
+constexpr int kRingV = 5;                                // V halves in flight
+constexpr int kSplit = 4;                                // softmax threads per query row (32 key columns each)
 constexpr int kSBuf = 3;                                 // S/P buffers in TMEM
 constexpr int kPvRing = 4;                               // barriers that count completed P V products
-constexpr int kThreads = 384;                            // 3 warpgroups
+constexpr int kThreads = 128 + kSplit * 128;             // producers + MMA issuers, then kSplit softmax warpgroups
 constexpr uint32_t kSubTileBytes = 128 * 128;            // [128 rows x 64 bf16], 16 KiB
 constexpr uint32_t kTileBytes = 2 * kSubTileBytes;       // 32 KiB: the Q tile, or a whole K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;          // 16 KiB: what one CTA holds of a K or V tile
 constexpr uint32_t kKSubBytes = 64 * 128;                // [64 keys x 64 channels] sub-tile of a K half
-constexpr uint32_t kSmemTiles = kTileBytes + 2 * kRing * kHalfBytes;
-constexpr int kNumBars = 1 + 4 * kRing + 2 * kSBuf + kPvRing + 1;
+constexpr uint32_t kSmemTiles = kTileBytes + (kRing + kRingV) * kHalfBytes;
+constexpr int kNumBars = 1 + 2 * kRing + 2 * kRingV + 2 * kSBuf + kPvRing + 1;
 constexpr uint32_t kBarBytes = 384;                      // barriers, TMEM slot, abort flag
-constexpr uint32_t kXchgBytes = 2 * 2 * 128 * 4;         // [tile parity][column half][row] floats
+constexpr uint32_t kXchgBytes = 2 * kSplit * 128 * 4;    // [tile parity][column quarter][row] floats
 constexpr uint32_t kSmemNeeded = kSmemTiles + kBarBytes + kXchgBytes;
 constexpr uint32_t kSmemBytes = 227 * 1024;              // everything an SM offers one CTA
 static_assert(8 * kNumBars + 16 <= kBarBytes, "barrier area too small");
@@ -117,16 +121,16 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   auto bar_kfull = [&](int s) { return bars + 8u * (1 + s); };
   auto bar_kempty = [&](int s) { return bars + 8u * (1 + kRing + s); };
   auto bar_vfull = [&](int s) { return bars + 8u * (1 + 2 * kRing + s); };
-  auto bar_vempty = [&](int s) { return bars + 8u * (1 + 3 * kRing + s); };
-  auto bar_sfull = [&](int b) { return bars + 8u * (1 + 4 * kRing + b); };
-  auto bar_pfull = [&](int b) { return bars + 8u * (1 + 4 * kRing + kSBuf + b); };
-  auto bar_pvdone = [&](int i) { return bars + 8u * (1 + 4 * kRing + 2 * kSBuf + i); };
+  auto bar_vempty = [&](int s) { return bars + 8u * (1 + 2 * kRing + kRingV + s); };
+  auto bar_sfull = [&](int b) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + b); };
+  auto bar_pfull = [&](int b) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + kSBuf + b); };
+  auto bar_pvdone = [&](int i) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + 2 * kSBuf + i); };
   const uint32_t bar_done = bars + 8u * (kNumBars - 1);
   unsigned char* base_generic = smem_raw + (base - raw);
   unsigned char* bars_generic = base_generic + kSmemTiles;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * kNumBars + 8);
-  float* xchg = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [2][2][128]
+  float* xchg = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [2][kSplit][128]
 
   const int h = blockIdx.x, mt = blockIdx.y, unit = blockIdx.z;      // the pair = heads (h & ~1, h | 1)
   const uint32_t rank = cluster_rank();                               // 0 = leader
@@ -163,11 +167,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   if (tid == 0) {
     if (bad || misaligned) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
     mbar_init(bar_q, 1);
-    for (int s = 0; s < kRing; ++s) {
-      mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
-      mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
-    }
-    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 16); }
+    for (int s = 0; s < kRing; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
+    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); }
+    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 2 * kSplit * 4); }
     for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
     mbar_init(bar_done, 1);
     *abort_flag = 0;
@@ -214,8 +216,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     int page_cur = 0, page_next = resolve(0);
     bool ok = true;
     int issued = 0;
+    const int ring_n = is_v ? kRingV : kRing;
     for (int j = 0; j < n_tiles && ok; ++j) {
-      const int s = j % kRing, it = j / kRing;
+      const int s = j % ring_n, it = j / ring_n;
       if ((j & 3) == 0) page_cur = page_next;
       const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + my_granule);
       if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
@@ -247,114 +250,104 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     // out the worst-case copy time instead
     if (!ok) {
       if (leader) {
-        for (int j = max(0, issued - kRing); j < issued; ++j) {
-          const uint32_t fl = is_v ? bar_vfull(j % kRing) : bar_kfull(j % kRing);
-          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(fl, (j / kRing) & 1); ++i) {}
+        for (int j = max(0, issued - ring_n); j < issued; ++j) {
+          const uint32_t fl = is_v ? bar_vfull(j % ring_n) : bar_kfull(j % ring_n);
+          for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(fl, (j / ring_n) & 1); ++i) {}
         }
         if (!is_v) for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
       } else {
         __nanosleep(200000);
       }
     }
-  } else if (warp == 1) {
-    // =========================== MMA issuer ===========================
+  } else if (warp == 1 || warp == 3) {
+    // =========================== MMA issuers (leader CTA): warp 1 -> S = Q K^T, warp 3 -> O += P V ===========================
+    // Two issuing threads, so that a wait of one product (a late K tile; P not yet published) does
+    // not stop the issue of the other: a thread that issues tcgen05.mma is held back to the pipe's
+    // pace, and whatever it waits for in between leaves the pipe idle.  Products of different
+    // threads are not ordered by the pipe, so the reuse of an S/P buffer is ordered explicitly:
+    // QK(j) waits until PV(j - kSBuf), which read that buffer, has completed.
     if (lane == 0 && leader) {
-      constexpr uint32_t idesc_qk = make_idesc(false, 2 * kBM, kBN);
-      constexpr uint32_t idesc_pv = make_idesc(true, 2 * kBM, kBN);
-      const uint32_t tmem_o = tmem + kSBuf * 128;
-      // operand descriptors: high words are constants, low words advance by constant steps
-      constexpr uint32_t kHi = desc_hi(1024u);
-      const uint32_t q_lo = desc_lo(q_smem, 16u);
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
-      auto issue_qk = [&](int j) {                 // K(j) has landed
-        const int s = j % kRing;
-        tc_fence_after();
-        const uint32_t k_lo = desc_lo(k_ring + s * kHalfBytes, 16u);
-        const uint32_t s_tmem = tmem + (j % kSBuf) * 128;
-        // A: this CTA's 128 query rows; B: this CTA's 64 keys; both advance 16 channels per step
-        mma2_ss<false>(s_tmem, q_lo, k_lo, kHi, idesc_qk);
+      constexpr uint32_t kHi = desc_hi(1024u);       // descriptor high words are constants
+      bool ok = true;
+      if (warp == 1) {
+        constexpr uint32_t idesc_qk = make_idesc(false, 2 * kBM, kBN);
+        const uint32_t q_lo = desc_lo(q_smem, 16u);
+        ok = mbar_wait(bar_q, 0, abort_flag);
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const int s = j % kRing;
+          if (j >= kSBuf) ok = mbar_wait(bar_pvdone((j - kSBuf) % kPvRing), ((j - kSBuf) / kPvRing) & 1, abort_flag);
+          ok = ok && mbar_wait(bar_kfull(s), (j / kRing) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_lo = desc_lo(k_ring + s * kHalfBytes, 16u);
+          const uint32_t s_tmem = tmem + (j % kSBuf) * 128;
+          // A: this CTA's 128 query rows; B: this CTA's 64 keys; both advance 16 channels per step
+          mma2_ss<false>(s_tmem, q_lo, k_lo, kHi, idesc_qk);
 #pragma unroll
-        for (int k = 1; k < kD / 16; ++k) {
-          constexpr uint32_t kUnit = 16;     // descriptor addresses count 16-byte units
-          const uint32_t a_off = ((k >> 2) * kSubTileBytes + (k & 3) * 32u) / kUnit;
-          const uint32_t b_off = ((k >> 2) * kKSubBytes + (k & 3) * 32u) / kUnit;
-          mma2_ss<true>(s_tmem, q_lo + a_off, k_lo + b_off, kHi, idesc_qk);
+          for (int k = 1; k < kD / 16; ++k) {
+            constexpr uint32_t kUnit = 16;     // descriptor addresses count 16-byte units
+            const uint32_t a_off = ((k >> 2) * kSubTileBytes + (k & 3) * 32u) / kUnit;
+            const uint32_t b_off = ((k >> 2) * kKSubBytes + (k & 3) * 32u) / kUnit;
+            mma2_ss<true>(s_tmem, q_lo + a_off, k_lo + b_off, kHi, idesc_qk);
+          }
+          tc2_commit(bar_kempty(s));
+          tc2_commit(bar_sfull(j % kSBuf));
         }
-        tc2_commit(bar_kempty(s));
-        tc2_commit(bar_sfull(j % kSBuf));
-      };
-      auto issue_pv = [&](int i) {                 // V(i) has landed and both CTAs published P(i)
-        const int s = i % kRing, b = i % kSBuf;
-        tc_fence_after();
-        const uint32_t v_lo = desc_lo(v_ring + s * kHalfBytes, kSubTileBytes);
-        const uint32_t p_tmem = tmem + b * 128;
+      } else {
+        constexpr uint32_t idesc_pv = make_idesc(true, 2 * kBM, kBN);
+        const uint32_t tmem_o = tmem + kSBuf * 128;
+        for (int i = 0; i < n_tiles && ok; ++i) {
+          const int s = i % kRingV, b = i % kSBuf;
+          ok = mbar_wait(bar_vfull(s), (i / kRingV) & 1, abort_flag);
+          ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t v_lo = desc_lo(v_ring + s * kHalfBytes, kSubTileBytes);
+          const uint32_t p_tmem = tmem + b * 128;
 #pragma unroll
-        for (int k = 0; k < kBN / 16; ++k) {
-          // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
-          // term, then the 8 columns of the lo term of the same keys against the same V rows.
-          const uint32_t b_lo = v_lo + k * (2048u / 16u);
-          const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
-          mma2_ts(tmem_o, pa, b_lo, kHi, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
-          mma2_ts(tmem_o, pa + 16, b_lo, kHi, idesc_pv, 1u);
+          for (int k = 0; k < kBN / 16; ++k) {
+            // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
+            // term, then the 8 columns of the lo term of the same keys against the same V rows.
+            const uint32_t b_lo = v_lo + k * (2048u / 16u);
+            const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
+            mma2_ts(tmem_o, pa, b_lo, kHi, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
+            mma2_ts(tmem_o, pa + 16, b_lo, kHi, idesc_pv, 1u);
+          }
+          tc2_commit(bar_vempty(s));
+          tc2_commit(bar_pvdone(i % kPvRing));
         }
-        tc2_commit(bar_vempty(s));
-        tc2_commit(bar_pvdone(i % kPvRing));
-      };
-      // Whichever product has its operands is issued next: S = Q K^T may run up to kSBuf tiles
-      // ahead of O += P V (QK(j) reuses the buffer PV(j - kSBuf) read, and the pipe executes in
-      // issue order), so a late K tile does not hold back a ready P V, nor the reverse.
-      int qk = 0, pv = 0;
-      uint32_t idle = 0;
-      while (pv < n_tiles && ok) {
-        bool progressed = false;
-        const bool qk_allowed = qk < n_tiles && qk < pv + kSBuf;
-        if (qk_allowed && mbar_try_wait(bar_kfull(qk % kRing), (qk / kRing) & 1)) {
-          issue_qk(qk);
-          ++qk;
-          progressed = true;
-        }
-        if (pv < qk && mbar_try_wait(bar_vfull(pv % kRing), (pv / kRing) & 1) &&
-            mbar_try_wait(bar_pfull(pv % kSBuf), (pv / kSBuf) & 1)) {
-          issue_pv(pv);
-          ++pv;
-          progressed = true;
-        }
-        if (progressed) {
-          idle = 0;
-        } else if (++idle >= kSpinLimit || ((idle & 1023u) == 0 && *abort_flag)) {
-          *abort_flag = 1;
-          ok = false;
-        }
+        if (ok) tc2_commit(bar_done);      // the last P V depends, through the softmax, on every Q K^T
       }
-      if (ok) tc2_commit(bar_done);
     }
     __syncwarp();
   } else if (warp >= 4) {
     // =========================== softmax / epilogue ===========================
-    const int b = (warp >> 2) - 1;                        // column half of every tile
+    // A query row (= TMEM lane) is shared by kSplit threads, 32 key columns each; the four warps
+    // of a lane quadrant sit on the same scheduler, so their stalls overlap.
+    const int cq = (warp >> 2) - 1;                       // column quarter of every tile
     const int q4 = warp & 3;                              // TMEM lane quadrant of this warp
     const int row = q4 * 32 + lane;                       // query row inside the tile
     const uint32_t lane_addr = uint32_t(q4 * 32) << 16;
-    const uint32_t o_addr = tmem + lane_addr + kSBuf * 128 + b * 64;
+    const uint32_t o_addr = tmem + lane_addr + kSBuf * 128 + cq * 32;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
       const int sb = j % kSBuf;
       ok = ok && mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
       tc_fence_after();
-      const uint32_t s_addr = tmem + lane_addr + sb * 128 + b * 64;
-      uint64_t sv[32];
-      TMEM_LD64P_WAIT(s_addr, sv);
+      const uint32_t s_addr = tmem + lane_addr + sb * 128 + cq * 32;
+      uint64_t sv[16];
+      TMEM_LD32P_WAIT(s_addr, sv);
       // key-validity limit: ragged last past tile, or the causal diagonal of the last tile
       int limit = kBN;
       if (j < past_tiles) limit = min(kBN, n_past - j * kBN);
       else if (j == n_tiles - 1) limit = row + 1;
-      limit -= b * 64;                                    // in this thread's column numbering
+      limit -= cq * 32;                                   // in this thread's column numbering
       const bool masked = (j == n_tiles - 1) || (j == past_tiles - 1 && (n_past % kBN) != 0);   // CTA-uniform
       float mx = -INFINITY, mx2 = -INFINITY;
       if (masked) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
+        for (int i = 0; i < 16; ++i) {
           const float x0 = 2 * i < limit ? lo2(sv[i]) : -INFINITY;
           const float x1 = 2 * i + 1 < limit ? hi2(sv[i]) : -INFINITY;
           sv[i] = pack2(x0, x1);
@@ -363,7 +356,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       } else {
         float mx3 = -INFINITY, mx4 = -INFINITY;           // four independent chains
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
+        for (int i = 0; i < 16; i += 4) {
           mx = max3(mx, lo2(sv[i]), hi2(sv[i]));
           mx2 = max3(mx2, lo2(sv[i + 1]), hi2(sv[i + 1]));
           mx3 = max3(mx3, lo2(sv[i + 2]), hi2(sv[i + 2]));
@@ -371,12 +364,12 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
         mx = fmaxf(max3(mx, mx2, mx3), mx4);
       }
-      // the row's maximum over both column halves
-      float* xrow = xchg + (j & 1) * 256 + row;
-      xrow[b * 128] = mx;
-      ok = pair_sync_and(q4, ok);
-      if (!ok) break;                                     // both threads of a row leave together
-      mx = fmaxf(mx, xrow[(1 - b) * 128]);
+      // the row's maximum over the four column quarters
+      float* xrow = xchg + (j & 1) * (kSplit * 128) + row;
+      xrow[cq * 128] = mx;
+      ok = quadrant_sync_and<kSplit>(q4, ok);
+      if (!ok) break;                                     // the threads of a row leave together
+      mx = fmaxf(fmaxf(xrow[0], xrow[128]), fmaxf(xrow[256], xrow[384]));
       const float m_new = fmaxf(m_used, mx * p.scale_log2);
       const bool grow = m_new - m_used > kRescaleThreshold;     // also true for the first tile
       if (j == 0) {
@@ -389,80 +382,71 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tc_fence_after();
         const float f = grow ? ex2(m_used - m_new) : 1.f;
         if (grow) { m_used = m_new; l *= f; }
+        uint32_t orr[32];
+        TMEM_LD32_WAIT(o_addr, orr);
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          uint32_t orr[32];
-          TMEM_LD32_WAIT(o_addr + cc * 32, orr);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
-          TMEM_ST32(o_addr + cc * 32, orr);
-        }
+        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
+        TMEM_ST32(o_addr, orr);
       }
       // P = exp2(x - m) split into two bf16 terms (hi + lo): with outlier value channels a
       // single bf16 P (8 significant bits) would cost up to |v| * 2^-9 of absolute error.
       const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm2 = pack2(-m_used, -m_used);
       uint64_t sum_a = 0, sum_b = 0;                      // two (+0, +0) pairs
+      uint32_t pk[32];
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        uint32_t pk[32];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint64_t x = fma2(sv[16 * cc + i], scale2, negm2);
-          const float e0 = ex2(lo2(x)), e1 = ex2(hi2(x));
-          const uint64_t e = pack2(e0, e1);
-          if (i & 1) sum_b = add2(sum_b, e); else sum_a = add2(sum_a, e);
-          const uint32_t hi = pack_bf16(e0, e1);
-          pk[i] = hi;
-          const uint64_t lo = sub2(e, (uint64_t(hi & 0xFFFF0000u) << 32) | (hi << 16));
-          pk[16 + i] = pack_bf16(lo2(lo), hi2(lo));
-        }
-        TMEM_ST32(s_addr + cc * 32, pk);
+      for (int i = 0; i < 16; ++i) {
+        const uint64_t x = fma2(sv[i], scale2, negm2);
+        const float e0 = ex2(lo2(x)), e1 = ex2(hi2(x));
+        const uint64_t e = pack2(e0, e1);
+        if (i & 1) sum_b = add2(sum_b, e); else sum_a = add2(sum_a, e);
+        const uint32_t hi = pack_bf16(e0, e1);
+        pk[i] = hi;
+        const uint64_t lo = sub2(e, (uint64_t(hi & 0xFFFF0000u) << 32) | (hi << 16));
+        pk[16 + i] = pack_bf16(lo2(lo), hi2(lo));
       }
+      TMEM_ST32(s_addr, pk);
       sum_a = add2(sum_a, sum_b);
       l += lo2(sum_a) + hi2(sum_a);
       tmem_wait_st();
       tc_fence_before();
-      __syncwarp();                                       // one arrival per warp: 8 warps in each CTA
+      __syncwarp();                                       // one arrival per warp: 32 of both CTAs' warps in all
       if (lane == 0) mbar_arrive_cluster(leader_addr(bar_pfull(sb)));
     }
-    // ---- epilogue: the row sum over both column halves, then this thread's 64 channels of O / l
+    // ---- epilogue: the row sum over the four column quarters, then this thread's 32 channels of O / l
     ok = ok && mbar_wait(bar_done, 0, abort_flag);
-    float* xrow = xchg + (n_tiles & 1) * 256 + row;
-    xrow[b * 128] = l;
-    ok = pair_sync_and(q4, ok);
+    float* xrow = xchg + (n_tiles & 1) * (kSplit * 128) + row;
+    xrow[cq * 128] = l;
+    ok = quadrant_sync_and<kSplit>(q4, ok);
     if (ok) {
       tc_fence_after();
-      const float lsum = l + xrow[(1 - b) * 128];
+      const float lsum = (xrow[0] + xrow[128]) + (xrow[256] + xrow[384]);
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
       const size_t tok = size_t(unit) * nt + size_t(mt) * kBM + row;
+      const int col = cq * 32;
+      uint32_t orr[32];
+      TMEM_LD32_WAIT(o_addr, orr);
+      if (p.out_bf16) {
+        __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        const int col = b * 64 + cc * 32;
-        uint32_t orr[32];
-        TMEM_LD32_WAIT(o_addr + cc * 32, orr);
-        if (p.out_bf16) {
-          __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
+        for (int i = 0; i < 4; ++i) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
+          v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
+          v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
+          v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+          *reinterpret_cast<uint4*>(ob + 8 * i) = v;
+        }
+      } else {
+        float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 v;
-            v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
-            v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
-            v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
-            v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
-            *reinterpret_cast<uint4*>(ob + 8 * i) = v;
-          }
-        } else {
-          float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float4 v;
-            v.x = __uint_as_float(orr[4 * i + 0]) * inv; v.y = __uint_as_float(orr[4 * i + 1]) * inv;
-            v.z = __uint_as_float(orr[4 * i + 2]) * inv; v.w = __uint_as_float(orr[4 * i + 3]) * inv;
-            *reinterpret_cast<float4*>(of + 4 * i) = v;
-          }
+        for (int i = 0; i < 8; ++i) {
+          float4 v;
+          v.x = __uint_as_float(orr[4 * i + 0]) * inv; v.y = __uint_as_float(orr[4 * i + 1]) * inv;
+          v.z = __uint_as_float(orr[4 * i + 2]) * inv; v.w = __uint_as_float(orr[4 * i + 3]) * inv;
+          *reinterpret_cast<float4*>(of + 4 * i) = v;
         }
       }
-      if (p.a.lse && b == 0)
+      if (p.a.lse && cq == 0)
         p.a.lse[(size_t(unit) * p.n_q_heads + h) * nt + size_t(mt) * kBM + row] =
             (m_used + log2f(lsum)) * 0.6931471805599453f;
     }

@@ -329,6 +329,7 @@ int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaS
     if (smem > 220 * 1024) return ACTQKV_ERR_SHAPE;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
       return ACTQKV_ERR_LAUNCH;
+    prefer_max_shared(kern);
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(split, cfg->n_q_heads, b.units());
     lc.blockDim = dim3(kThreads, 1, 1);

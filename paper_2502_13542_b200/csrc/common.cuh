@@ -50,6 +50,14 @@ inline size_t elt_size(const actqkv_config* c) { return c->dtype == ACTQKV_BF16 
     if ((p) && !actqkv::aligned16(p)) return ACTQKV_ERR_ALIGN; \
   } while (0)
 
+// Every kernel of the library asks for the largest shared-memory carve-out, as the attention
+// kernels need: consecutive kernels of a step then run under one L1 / shared-memory split and
+// the SMs are not reconfigured between them.
+template <typename Kernel>
+inline void prefer_max_shared(Kernel kern) {
+  (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, int(cudaSharedmemCarveoutMaxShared));
+}
+
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? ACTQKV_OK : ACTQKV_ERR_LAUNCH; }
 
 // ---------------------------------------------------------------- device helpers

@@ -151,6 +151,8 @@ void launch_scores_t(const actqkv_config* cfg, const Batch& b, const float* prob
                      const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
                      cudaStream_t st) {
   dim3 grid((cfg->n_cap + kBlocksPerCta - 1) / kBlocksPerCta, cfg->n_kv_heads, b.units());
+  prefer_max_shared(score_kernel<T, D, false>);
+  prefer_max_shared(score_kernel<T, D, true>);
   if (cfg->agg_mode == ACTQKV_AGG_MAX)
     score_kernel<T, D, false><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
                                                               n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
@@ -194,6 +196,7 @@ extern "C" int actqkv_score_blocks(const actqkv_config* cfg, const actqkv_batch*
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   rc = launch_scores(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
   if (rc) return rc;
+  prefer_max_shared(entropy_kernel);
   entropy_kernel<<<dim3(cfg->n_kv_heads, b.units()), 32, 0, st>>>(
       scores, n_cand, theta, cfg->n_kv_heads, cfg->n_cap, b.n_layers, cfg->beta);
   return launch_status();

@@ -335,10 +335,12 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
     const size_t sm_chain = sizeof(float) * ((size_t(b.n_layers) * cfg->n_kv_heads + 1) & ~size_t(1)) +
                             sizeof(double) * 2 * (size_t(cfg->n_layers) + 1);
     if (sm_chain > 48 * 1024) return ACTQKV_ERR_SHAPE;
+    prefer_max_shared(cutoff_chain_kernel);
     cutoff_chain_kernel<<<b.n_seq, kChainThreads, sm_chain, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;
     if (cfg->cap_blocks == 0) return ACTQKV_OK;
   }
+  prefer_max_shared(kern);
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(cfg->n_kv_heads, b.units(), 1);
   lc.blockDim = dim3(kSelThreads, 1, 1);
