@@ -25,7 +25,8 @@ template <typename T, int D, bool kMean>
 __global__ void __launch_bounds__(kScoreThreads)
 score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
              const float* __restrict__ repr_inv_norm, const int32_t* __restrict__ n_cand,
-             float* __restrict__ scores, int n_kv_heads, int r, int n_cap, int n_layers, int32_t* status) {
+             float* __restrict__ scores, int n_kv_heads, int r, int n_cap, int n_layers, int groups,
+             int32_t* status) {
   const int g = blockIdx.y, unit = blockIdx.z;
   const int seq = unit / n_layers;
   int n = n_cand[seq];
@@ -34,7 +35,8 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
     if (threadIdx.x == 0 && blockIdx.x == 0 && g == 0) set_status(status, ACTQKV_DEV_NCAND_CLAMPED);
   }
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b0 = (blockIdx.x * (kScoreThreads / 32) + warp) * kBlocksPerWarp;
+  // a warp scores `groups` groups of kBlocksPerWarp consecutive blocks
+  const int b0 = (blockIdx.x * (kScoreThreads / 32) + warp) * kBlocksPerWarp * groups;
   if (b0 >= n) return;                    // warp-uniform; no block-wide barrier below
 
   constexpr int VN = Vec16<T>::N;
@@ -43,22 +45,30 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
   const int sub = lane / LPR, lir = lane - sub * LPR;
   const size_t head_rows = (size_t(unit) * n_kv_heads + g) * size_t(n_cap) * r;
   const int n_pass = (r + RPP - 1) / RPP;
-  const T* tab0 = repr_k + (head_rows + size_t(b0) * r) * D + lir * VN;
-  const float* inv0 = repr_inv_norm + head_rows + size_t(b0) * r;
+  const T* tab = repr_k + head_rows * D + lir * VN;
+  const float* inv = repr_inv_norm + head_rows;
 
-  // every row of the warp's blocks first (independent 16-byte loads), then the probe
-  uint4 kv[kBlocksPerWarp][kMaxPasses];             // raw 16-byte vectors, unpacked at use
-  float nrm[kBlocksPerWarp][kMaxPasses];
+  // One group's rows: raw 16-byte vectors (unpacked at use) and the rows' inverse norms.
+  struct Group {
+    uint4 kv[kBlocksPerWarp][kMaxPasses];
+    float nrm[kBlocksPerWarp][kMaxPasses];
+  };
+  auto load_group = [&](int bg, Group& gr) {
 #pragma unroll
-  for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
+    for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
 #pragma unroll
-    for (int ps = 0; ps < kMaxPasses; ++ps) {
-      const int i = ps * RPP + sub;
-      const bool on = b0 + bi < n && i < r;
-      nrm[bi][ps] = on ? __ldg(inv0 + bi * r + i) : 0.f;
-      kv[bi][ps] = on ? __ldg(reinterpret_cast<const uint4*>(tab0 + (size_t(bi) * r + i) * D)) : make_uint4(0, 0, 0, 0);
+      for (int ps = 0; ps < kMaxPasses; ++ps) {
+        const int i = ps * RPP + sub;
+        const bool on = bg + bi < n && i < r;
+        const size_t row = size_t(bg + bi) * r + i;
+        gr.nrm[bi][ps] = on ? __ldg(inv + row) : 0.f;
+        gr.kv[bi][ps] = on ? __ldg(reinterpret_cast<const uint4*>(tab + row * D)) : make_uint4(0, 0, 0, 0);
+      }
     }
-  }
+  };
+  // the first group's loads go out before anything else, then the probe
+  Group ga, gb;
+  load_group(b0, ga);
   const float* pg = probe_kv + (size_t(unit) * n_kv_heads + g) * D;
   float pv[VN];
   Vec16<float>::load_nc(pg + lir * VN, reinterpret_cast<float(&)[4]>(pv[0]));
@@ -74,62 +84,73 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
   const float inv_pn = bad ? 0.f : rsqrtf(sq);
   float* out = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
 
+  auto score_group = [&](int bg, const Group& gr) {
 #pragma unroll
-  for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
-    const int b = b0 + bi;
-    if (b >= n) break;                    // warp-uniform
-    if constexpr (kMean) {
-      float acc = 0.f;                    // sum over this lane's rows of (partial dot) / ||R_i||
-      for (int p0 = 0; p0 < n_pass; p0 += kMaxPasses) {
+    for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
+      const int b = bg + bi;
+      if (b >= n) break;                  // warp-uniform
+      if constexpr (kMean) {
+        float acc = 0.f;                  // sum over this lane's rows of (partial dot) / ||R_i||
+        for (int p0 = 0; p0 < n_pass; p0 += kMaxPasses) {
 #pragma unroll
-        for (int ps = 0; ps < kMaxPasses; ++ps) {
-          float row[VN];
-          float w = nrm[bi][ps];
-          if (p0 == 0) {
-            Vec16<T>::unpack(kv[bi][ps], row);
-          } else {                        // more row groups than the registers hold
-            const int i = (p0 + ps) * RPP + sub;
-            w = 0.f;
+          for (int ps = 0; ps < kMaxPasses; ++ps) {
+            float row[VN];
+            float w = gr.nrm[bi][ps];
+            if (p0 == 0) {
+              Vec16<T>::unpack(gr.kv[bi][ps], row);
+            } else {                      // more row groups than the registers hold
+              const int i = (p0 + ps) * RPP + sub;
+              w = 0.f;
 #pragma unroll
-            for (int e = 0; e < VN; ++e) row[e] = 0.f;
-            if (i < r) {
-              w = __ldg(inv0 + bi * r + i);
-              Vec16<T>::load_nc(tab0 + (size_t(bi) * r + i) * D, row);
+              for (int e = 0; e < VN; ++e) row[e] = 0.f;
+              if (i < r) {
+                w = __ldg(inv + size_t(b) * r + i);
+                Vec16<T>::load_nc(tab + (size_t(b) * r + i) * D, row);
+              }
             }
+            float dot = 0.f;
+#pragma unroll
+            for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], row[e], dot);
+            acc = fmaf(dot, w, acc);
+          }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) out[b] = acc * inv_pn / float(r);
+      } else {
+        float agg = -INFINITY;
+        for (int ps = 0; ps < n_pass; ++ps) {
+          const int i = ps * RPP + sub;
+          float row[VN];
+          float w = 0.f;
+#pragma unroll
+          for (int e = 0; e < VN; ++e) row[e] = 0.f;
+          if (i < r) {
+            w = __ldg(inv + size_t(b) * r + i);
+            Vec16<T>::load_nc(tab + (size_t(b) * r + i) * D, row);
           }
           float dot = 0.f;
 #pragma unroll
           for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], row[e], dot);
-          acc = fmaf(dot, w, acc);
+#pragma unroll
+          for (int o = LPR >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          float cosv = i < r ? dot * inv_pn * w : -INFINITY;
+          // maximum over the row groups of this pass (group leaders hold the cosines)
+#pragma unroll
+          for (int o = LPR; o < 32; o <<= 1) cosv = fmaxf(cosv, __shfl_xor_sync(0xffffffffu, cosv, o));
+          agg = fmaxf(agg, cosv);
         }
+        if (lane == 0) out[b] = agg;
       }
-      acc = warp_sum(acc);
-      if (lane == 0) out[b] = acc * inv_pn / float(r);
-    } else {
-      float agg = -INFINITY;
-      for (int ps = 0; ps < n_pass; ++ps) {
-        const int i = ps * RPP + sub;
-        float row[VN];
-        float w = 0.f;
-#pragma unroll
-        for (int e = 0; e < VN; ++e) row[e] = 0.f;
-        if (i < r) {
-          w = __ldg(inv0 + bi * r + i);
-          Vec16<T>::load_nc(tab0 + (size_t(bi) * r + i) * D, row);
-        }
-        float dot = 0.f;
-#pragma unroll
-        for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], row[e], dot);
-#pragma unroll
-        for (int o = LPR >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        float cosv = i < r ? dot * inv_pn * w : -INFINITY;
-        // maximum over the row groups of this pass (group leaders hold the cosines)
-#pragma unroll
-        for (int o = LPR; o < 32; o <<= 1) cosv = fmaxf(cosv, __shfl_xor_sync(0xffffffffu, cosv, o));
-        agg = fmaxf(agg, cosv);
-      }
-      if (lane == 0) out[b] = agg;
     }
+  };
+  // double-buffered: the next group's loads are in flight while the current group is scored
+  for (int gi = 0; gi < groups; gi += 2) {
+    const int bg = b0 + gi * kBlocksPerWarp;
+    if (bg >= n) break;
+    if (gi + 1 < groups) load_group(bg + kBlocksPerWarp, gb);
+    score_group(bg, ga);
+    if (gi + 2 < groups) load_group(bg + 2 * kBlocksPerWarp, ga);
+    if (gi + 1 < groups) score_group(bg + kBlocksPerWarp, gb);
   }
 }
 
@@ -150,17 +171,24 @@ template <typename T, int D>
 void launch_scores_t(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,
                      const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
                      cudaStream_t st) {
-  dim3 grid((cfg->n_cap + kBlocksPerCta - 1) / kBlocksPerCta, cfg->n_kv_heads, b.units());
+  // blocks per warp: one group of kBlocksPerWarp when the call is small (latency matters, spread
+  // it over as many CTAs as possible), more groups (software-pipelined) once the grid would
+  // exceed a few CTAs per SM anyway
+  const int ctas_1 = (cfg->n_cap + kBlocksPerCta - 1) / kBlocksPerCta;
+  const long long total_1 = (long long)ctas_1 * cfg->n_kv_heads * b.units();
+  int groups = 1;
+  while (groups < 8 && total_1 / (2 * groups) >= 4 * 148 && ctas_1 / (2 * groups) >= 1) groups *= 2;
+  dim3 grid((cfg->n_cap + kBlocksPerCta * groups - 1) / (kBlocksPerCta * groups), cfg->n_kv_heads, b.units());
   prefer_max_shared(score_kernel<T, D, false>);
   prefer_max_shared(score_kernel<T, D, true>);
   if (cfg->agg_mode == ACTQKV_AGG_MAX)
     score_kernel<T, D, false><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
                                                               n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
-                                                              cfg->n_cap, b.n_layers, status);
+                                                              cfg->n_cap, b.n_layers, groups, status);
   else
     score_kernel<T, D, true><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
                                                              n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
-                                                             cfg->n_cap, b.n_layers, status);
+                                                             cfg->n_cap, b.n_layers, groups, status);
 }
 
 int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,
@@ -175,6 +203,14 @@ int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_k
     if (bf16) launch_scores_t<__nv_bfloat16, 128>(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
     else launch_scores_t<float, 128>(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
   }
+  return launch_status();
+}
+
+int launch_entropy(const actqkv_config* cfg, const Batch& b, const float* scores, const int32_t* n_cand,
+                   float* theta, cudaStream_t st) {
+  prefer_max_shared(entropy_kernel);
+  entropy_kernel<<<dim3(cfg->n_kv_heads, b.units()), 32, 0, st>>>(scores, n_cand, theta, cfg->n_kv_heads, cfg->n_cap,
+                                                                 b.n_layers, cfg->beta);
   return launch_status();
 }
 
@@ -196,8 +232,5 @@ extern "C" int actqkv_score_blocks(const actqkv_config* cfg, const actqkv_batch*
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   rc = launch_scores(cfg, b, probe_kv, repr_k, repr_inv_norm, n_cand, scores, status, st);
   if (rc) return rc;
-  prefer_max_shared(entropy_kernel);
-  entropy_kernel<<<dim3(cfg->n_kv_heads, b.units()), 32, 0, st>>>(
-      scores, n_cand, theta, cfg->n_kv_heads, cfg->n_cap, b.n_layers, cfg->beta);
-  return launch_status();
+  return launch_entropy(cfg, b, scores, n_cand, theta, st);
 }

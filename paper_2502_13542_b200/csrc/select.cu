@@ -69,51 +69,78 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
     if (lane == 0) theta_h[pair] = th;
   }
   __syncthreads();
-  if (threadIdx.x != 0) return;
 
+  // Shared work arrays after the densities: doubles [Lb] th, [L + 1] suffix of known theta-bars,
+  // [L + 1] suffix count of layers without one, [Lb] ratio.
+  double* th_l = reinterpret_cast<double*>(theta_h + ((p.Lb * p.n_kv_heads + 1) & ~1));
+  double* suf_known = th_l + p.Lb;
+  double* suf_open = suf_known + p.L + 1;
+  double* ratio = suf_open + p.L + 1;
   double* st = p.state + size_t(seq) * (1 + 2 * p.L);
   double* hist_sum = st + 1;
   double* hist_cnt = st + 1 + p.L;
-  double b_rem = st[0];
-  auto layer_theta = [&](int l) {
+  const int tid = threadIdx.x;
+  // ---- in parallel: each batched layer's density (mean over its KV heads, fixed order)
+  if (tid < p.Lb) {
     double s = 0.0;
-    for (int g = 0; g < p.n_kv_heads; ++g) s += double(theta_h[l * p.n_kv_heads + g]);
-    return s / double(p.n_kv_heads);
-  };
-  // Suffix sums over the deeper layers, so that the walk below is linear in L: `known` adds the
-  // theta-bar of the layers that have one (their history mean, or this call's own density in the
-  // Algorithm-1 reading), `open` counts the layers that take the current layer's density instead.
-  // suffix[l] covers layers > l of the MODEL (index = model layer); the batch holds layers
-  // layer0 .. layer0 + Lb - 1.
-  double* suf_known = reinterpret_cast<double*>(theta_h + ((p.Lb * p.n_kv_heads + 1) & ~1));   // [L + 1]
-  double* suf_open = suf_known + p.L + 1;                                                       // [L + 1]
-  suf_known[p.L] = 0.0;
-  suf_open[p.L] = 0.0;
-  for (int j = p.L - 1; j >= 0; --j) {
+    for (int g = 0; g < p.n_kv_heads; ++g) s += double(theta_h[tid * p.n_kv_heads + g]);
+    th_l[tid] = s / double(p.n_kv_heads);
+  }
+  __syncthreads();
+  // ---- in parallel: theta-bar of every model layer that has one (its history mean, or this call's
+  // own density in the Algorithm-1 reading); the others will take the current layer's density
+  if (tid < p.L) {
     double known = 0.0, open = 0.0;
-    if (p.thetabar_mode == ACTQKV_THETABAR_ALG1) known = layer_theta(j - p.layer0);
-    else if (hist_cnt[j] > 0.0) known = hist_sum[j] / hist_cnt[j];
+    if (p.thetabar_mode == ACTQKV_THETABAR_ALG1) known = th_l[tid - p.layer0];
+    else if (hist_cnt[tid] > 0.0) known = hist_sum[tid] / hist_cnt[tid];
     else open = 1.0;
-    suf_known[j] = suf_known[j + 1] + known;
-    suf_open[j] = suf_open[j + 1] + open;
+    suf_known[tid] = known;          // turned into suffix sums below
+    suf_open[tid] = open;
   }
-  for (int l = 0; l < p.Lb; ++l) {
-    const int layer = p.layer0 + l;
-    if (layer == 0) b_rem = double(p.L) * double(p.k_blocks);
-    const double th = layer_theta(l);
-    Grant gr{0, 0.0};
-    if (n > 0) {
-      const double rest = suf_known[layer + 1] + suf_open[layer + 1] * th;
-      gr = grant_layer(th, rest, b_rem, p.L - layer, n, p.cap_blocks);
-      b_rem -= double(gr.c);
-      hist_sum[layer] += th;
-      hist_cnt[layer] += 1.0;
+  __syncthreads();
+  if (tid == 0) {                    // suffix[j] = sum over layers >= j (additions only)
+    suf_known[p.L] = 0.0;
+    suf_open[p.L] = 0.0;
+    for (int j = p.L - 1; j >= 0; --j) {
+      suf_known[j] += suf_known[j + 1];
+      suf_open[j] += suf_open[j + 1];
     }
-    const size_t unit = size_t(seq) * p.Lb + l;
-    p.sel_count[unit] = gr.c;
-    if (p.budget_real) p.budget_real[unit] = float(gr.real);
   }
-  st[0] = b_rem;
+  __syncthreads();
+  // ---- in parallel: the share theta / (theta + sum of deeper theta-bars) of Eq. 12, which does
+  // not depend on the running budget
+  if (tid < p.Lb) {
+    const int layer = p.layer0 + tid;
+    const double th = th_l[tid];
+    const double den = th + suf_known[layer + 1] + suf_open[layer + 1] * th;
+    ratio[tid] = den > 0.0 ? th / den : -1.0;
+  }
+  __syncthreads();
+  // ---- serial: the budget walks the layers shallow -> deep
+  if (tid == 0) {
+    double b_rem = st[0];
+    for (int l = 0; l < p.Lb; ++l) {
+      const int layer = p.layer0 + l;
+      if (layer == 0) b_rem = double(p.L) * double(p.k_blocks);
+      int c = 0;
+      double real = 0.0;
+      if (n > 0) {
+        real = ratio[l] >= 0.0 ? ratio[l] * b_rem : b_rem / double(p.L - layer);
+        const double fl = floor(real + 0.5);
+        c = fl > 2.0e9 ? 2000000000 : (fl < -2.0e9 ? -2000000000 : int(fl));
+        c = max(min(1, n), min(c, min(p.cap_blocks, n)));
+        b_rem -= double(c);
+      }
+      const size_t unit = size_t(seq) * p.Lb + l;
+      p.sel_count[unit] = c;
+      if (p.budget_real) p.budget_real[unit] = float(real);
+    }
+    st[0] = b_rem;
+  }
+  if (tid < p.Lb && n > 0) {         // density history of the layers of this call
+    hist_sum[p.layer0 + tid] += th_l[tid];
+    hist_cnt[p.layer0 + tid] += 1.0;
+  }
 }
 
 // Order-preserving key: larger score <-> larger unsigned key; NaN lowest; -0 == +0.
@@ -333,8 +360,14 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
     return ACTQKV_ERR_LAUNCH;
   if (!fused) {
     const size_t sm_chain = sizeof(float) * ((size_t(b.n_layers) * cfg->n_kv_heads + 1) & ~size_t(1)) +
-                            sizeof(double) * 2 * (size_t(cfg->n_layers) + 1);
+                            sizeof(double) * (2 * size_t(b.n_layers) + 2 * (size_t(cfg->n_layers) + 1));
     if (sm_chain > 48 * 1024) return ACTQKV_ERR_SHAPE;
+    if (!p.theta_in && theta_out && b.n_layers * cfg->n_kv_heads >= 64) {
+      // many (layer, head) densities: take them with one warp each in a kernel of their own
+      const int rc = launch_entropy(cfg, b, scores, n_cand, theta_out, st);
+      if (rc) return rc;
+      p.theta_in = theta_out;
+    }
     prefer_max_shared(cutoff_chain_kernel);
     cutoff_chain_kernel<<<b.n_seq, kChainThreads, sm_chain, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;

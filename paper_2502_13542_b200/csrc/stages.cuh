@@ -28,6 +28,10 @@ int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_k
                   const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
                   cudaStream_t st);
 
+// Eq. 11 for every (unit, KV head), one warp each.
+int launch_entropy(const actqkv_config* cfg, const Batch& b, const float* scores, const int32_t* n_cand,
+                   float* theta, cudaStream_t st);
+
 // Retrieval attention kernels: the general fp32-accumulate kernel and the tcgen05 kernel.
 struct AttnArgs {
   const void *q, *k_win, *v_win, *k_pages, *v_pages;
