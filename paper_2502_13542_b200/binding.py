@@ -283,10 +283,22 @@ class RetrievalState:
         self.n_cand.copy_(torch.tensor(nc, dtype=torch.int32), non_blocking=False)
 
     def step(self, q, k_win, v_win, out, n_tokens=None, lse=None, fused=True, update_probe=True,
-             advance=True):
-        """bias -> probe -> score -> cut-off/select -> attention -> append for every unit."""
+             advance=True, overlap_append=False):
+        """bias -> probe -> score -> cut-off/select -> attention -> append for every unit.
+
+        overlap_append: enqueue the append on a second stream, concurrent with the other five
+        stages (it reads only the step's own K / V and writes pages and table rows that the other
+        stages of the same step do not read); the streams are joined before the step returns."""
         cfg, b = self.cfg, self.batch
         nt = n_tokens if n_tokens is not None else q.shape[-3]
+        main = torch.cuda.current_stream()
+        if overlap_append:
+            if getattr(self, "_side", None) is None:
+                self._side = torch.cuda.Stream(device=self.device)
+            self._side.wait_stream(main)
+            with torch.cuda.stream(self._side):
+                append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
+                              self.repr_k, self.repr_inv_norm, self.status)
         if update_probe:
             if fused:
                 bias_probe(cfg, b, q, nt, self.stats_count, self.stats_mean, self.stats_m2, self.phi_l1,
@@ -306,7 +318,10 @@ class RetrievalState:
                           self.sel_count, self.budget_real, self.status)
         retrieval_attention(cfg, b, q, k_win, v_win, nt, self.k_pages, self.v_pages, self.page_table,
                             self.pos0, self.sel_idx, self.sel_count, out, lse, self.status)
-        append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
-                      self.repr_k, self.repr_inv_norm, self.status)
+        if overlap_append:
+            main.wait_stream(self._side)
+        else:
+            append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
+                          self.repr_k, self.repr_inv_norm, self.status)
         if advance:
             self.set_positions([p + nt for p in self.host_pos0])
