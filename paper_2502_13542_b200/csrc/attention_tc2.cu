@@ -139,6 +139,26 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nt = p.a.n_tokens;
 
+  // ---- set-up that depends on no earlier kernel: barriers, TMEM
+  if (tid == 0) {
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < kRing; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
+    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); }
+    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 2 * kSplit * 4); }
+    for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
+    mbar_init(bar_done, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+  }
+  tc_fence_before();
+  cluster_sync_all();         // both CTAs' barriers are initialised and both hold their TMEM
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  grid_dependency_wait();            // the selection (and whatever produced Q / K / V) is complete from here on
   // ---- geometry (uniform over the CTA)
   const Geometry geo = make_geometry(p.a.pos0[seq], p.n_init, p.block, p.n_local_prev);
   int c = p.a.sel_count ? p.a.sel_count[unit] : 0;
@@ -164,25 +184,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   const int past_tiles = (n_past + kBN - 1) / kBN;
   const int n_tiles = past_tiles + mt + 1;
 
-  if (tid == 0) {
-    if (bad || misaligned) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
-    mbar_init(bar_q, 1);
-    for (int s = 0; s < kRing; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
-    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); }
-    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 2 * kSplit * 4); }
-    for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
-    mbar_init(bar_done, 1);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
-  }
-  tc_fence_before();
-  cluster_sync_all();         // both CTAs' barriers are initialised and both hold their TMEM
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  if (tid == 0 && (bad || misaligned)) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
   if (misaligned) {           // uniform over the pair: nothing was issued yet
     cluster_sync_all();
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
@@ -514,13 +516,14 @@ int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArg
   lc.blockDim = dim3(kThreads, 1, 1);
   lc.dynamicSmemBytes = kSmemBytes;
   lc.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  allow_early_launch(attr[1]);
   lc.attrs = attr;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
   if (cudaLaunchKernelEx(&lc, attention_tc2_kernel, tm_q, tm_kw, tm_vw, tm_kp, tm_vp, p) != cudaSuccess)
     return ACTQKV_ERR_LAUNCH;
   return launch_status();

@@ -82,6 +82,8 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams
   const size_t hd = (size_t(unit) * p.n_q_heads + h) * D;
   const size_t uh = size_t(unit) * p.n_q_heads + h;
 
+  grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
+  grid_launch_dependents();
   // ---- 0. rows -> shared memory: one bulk copy per row, all in flight together
   constexpr uint32_t kRowBytes = D * sizeof(T);
   const uint32_t bar_addr = smem_addr(bar);
@@ -335,13 +337,14 @@ int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaS
     lc.blockDim = dim3(kThreads, 1, 1);
     lc.dynamicSmemBytes = smem;
     lc.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = split;
     attr[0].val.clusterDim.y = cy;
     attr[0].val.clusterDim.z = 1;
+    allow_early_launch(attr[1]);
     lc.attrs = attr;
-    lc.numAttrs = 1;
+    lc.numAttrs = 2;
     if (cudaLaunchKernelEx(&lc, kern, p) == cudaSuccess) return launch_status();
     (void)cudaGetLastError();
   }

@@ -58,9 +58,22 @@ inline void prefer_max_shared(Kernel kern) {
   (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, int(cudaSharedmemCarveoutMaxShared));
 }
 
+// Programmatic dependent launch: a kernel launched with this attribute may start (run its
+// prologue: barrier set-up, loads of inputs no earlier kernel of the stream writes) while the
+// kernel before it in the stream is still draining; it must execute grid_dependency_wait()
+// before it touches anything an earlier kernel writes.  Without the attribute the wait is a no-op.
+inline void allow_early_launch(cudaLaunchAttribute& a) {
+  a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  a.val.programmaticStreamSerializationAllowed = 1;
+}
+
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? ACTQKV_OK : ACTQKV_ERR_LAUNCH; }
 
 // ---------------------------------------------------------------- device helpers
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream start its prologue; called after this kernel's own wait.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void set_status(int32_t* status, int bit) {
   if (status) atomicOr(status, bit);
 }

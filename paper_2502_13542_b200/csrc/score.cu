@@ -69,6 +69,8 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
   // the first group's loads go out before anything else, then the probe
   Group ga, gb;
   load_group(b0, ga);
+  grid_dependency_wait();            // the table is older than the stream's previous kernel; the probe is not
+  grid_launch_dependents();
   const float* pg = probe_kv + (size_t(unit) * n_kv_heads + g) * D;
   float pv[VN];
   Vec16<float>::load_nc(pg + lir * VN, reinterpret_cast<float(&)[4]>(pv[0]));
@@ -181,14 +183,21 @@ void launch_scores_t(const actqkv_config* cfg, const Batch& b, const float* prob
   dim3 grid((cfg->n_cap + kBlocksPerCta * groups - 1) / (kBlocksPerCta * groups), cfg->n_kv_heads, b.units());
   prefer_max_shared(score_kernel<T, D, false>);
   prefer_max_shared(score_kernel<T, D, true>);
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = dim3(kScoreThreads, 1, 1);
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  allow_early_launch(attr[0]);
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  const T* tab = static_cast<const T*>(repr_k);
   if (cfg->agg_mode == ACTQKV_AGG_MAX)
-    score_kernel<T, D, false><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
-                                                              n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
-                                                              cfg->n_cap, b.n_layers, groups, status);
+    (void)cudaLaunchKernelEx(&lc, score_kernel<T, D, false>, probe_kv, tab, repr_inv_norm, n_cand, scores,
+                             cfg->n_kv_heads, cfg->n_repr, cfg->n_cap, b.n_layers, groups, status);
   else
-    score_kernel<T, D, true><<<grid, kScoreThreads, 0, st>>>(probe_kv, static_cast<const T*>(repr_k), repr_inv_norm,
-                                                             n_cand, scores, cfg->n_kv_heads, cfg->n_repr,
-                                                             cfg->n_cap, b.n_layers, groups, status);
+    (void)cudaLaunchKernelEx(&lc, score_kernel<T, D, true>, probe_kv, tab, repr_inv_norm, n_cand, scores,
+                             cfg->n_kv_heads, cfg->n_repr, cfg->n_cap, b.n_layers, groups, status);
 }
 
 int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,

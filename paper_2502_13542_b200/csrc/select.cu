@@ -189,6 +189,8 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
   __shared__ float sh_theta;                   // this head's density (read by the cluster peers)
   __shared__ int sh_count;
   const int g = blockIdx.x, unit = blockIdx.y, tid = threadIdx.x;
+  grid_dependency_wait();            // scores / densities / counts come from the stream's previous kernels
+  grid_launch_dependents();
   const int n = min(n_cand[unit / n_layers], n_cap);
   const float* s = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
   int c;
@@ -379,13 +381,14 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
   lc.blockDim = dim3(kSelThreads, 1, 1);
   lc.dynamicSmemBytes = sm_sel;
   lc.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = fused ? cfg->n_kv_heads : 1;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  allow_early_launch(attr[1]);
   lc.attrs = attr;
-  lc.numAttrs = 1;
+  lc.numAttrs = fused ? 2 : 1;      // after the chain kernel (plain launch) the selection starts normally
   if (cudaLaunchKernelEx(&lc, kern, scores, n_cand, sel_count, sel_idx, cfg->n_kv_heads, cfg->n_cap,
                          cfg->cap_blocks, b.n_layers, status, p) != cudaSuccess)
     return ACTQKV_ERR_LAUNCH;
