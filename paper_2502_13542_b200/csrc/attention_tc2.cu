@@ -12,13 +12,24 @@
 // 32 KiB per tile instead of 64, and the rings hold 6 K halves and 5 V halves.  No TMA multicast
 // is used: each CTA fetches its own halves.
 //
-// Roles per CTA (640 threads): warp 0 K producer, warp 2 V producer, warps 1 and 3 the MMA issuers
+// Roles per CTA (768 threads): warp 0 K producer, warp 2 V producer, warps 1 and 3 the MMA issuers
 // (leader CTA = cluster rank 0 only; warp 1: S = Q K^T, warp 3: O += P V), warps 4-19 softmax with
 // FOUR threads per query row (32 key columns each; the four warps of a TMEM lane quadrant share a
-// scheduler, which hides their latencies).  Cross-CTA signalling:
-//   TMA loads of both CTAs complete on the LEADER's "full" barriers (cta_group::2 form of the load);
+// scheduler, which hides their latencies), warps 20-23 V conversion and O correction.
+//
+// P is kept in fp16 (11 significant bits; one tcgen05.mma per 16 keys, half the tensor-pipe time of
+// a bf16 high + low pair), so V must be fp16 too (kind::f16 wants both operands alike): warps 20-23
+// convert each CTA's half of a V tile in place after it landed, two tiles ahead of its use.  The row
+// sum adds the fp16-rounded P, so numerator and denominator carry the same rounding.  fp16 tops out
+// at 65504, so the running maximum used for P may lag the true one by at most 2^8; when it has to
+// move, O is rescaled by warps 20-23 between two P V products, off the softmax threads' path.
+// Cross-CTA signalling:
+//   K loads of both CTAs complete on the LEADER's "full" barriers (cta_group::2 form of the load);
+//   V loads complete on the loading CTA's barrier; its converter warps then arrive on the leader's
+//   "V ready" barrier;
 //   the leader's commits are multicast to the barriers of both CTAs (slot released, S ready, P V done);
-//   the softmax warps of both CTAs arrive on the leader's "P ready" barrier (one arrival per warp).
+//   the softmax warps of both CTAs arrive on the leader's "P ready" barrier (one arrival per warp),
+//   the correction warps on its "O corrected" barrier.
 // TMEM columns (both CTAs alike): S/P buffers 0..2 at [0,128) [128,256) [256,384), O at [384,512).
 // Every wait on an mbarrier is bounded; on expiry the CTA flags ACTQKV_DEV_TIMEOUT, stops issuing
 // work and drains; both CTAs meet at a cluster barrier before they free their TMEM.
@@ -32,18 +43,22 @@ namespace {
 constexpr int kBM = 128, kBN = 128, kD = 128;
 constexpr int kRing = 6;                                 // K halves in flight
 constexpr int kRingV = 5;                                // V halves in flight
+// fp16 P: exp2(x - m) must stay below 65504, so the running maximum may lag by at most 2^8
+constexpr float kRescaleF16 = 8.0f;
 constexpr int kSplit = 4;                                // softmax threads per query row (32 key columns each)
 constexpr int kSBuf = 3;                                 // S/P buffers in TMEM
 constexpr int kPvRing = 4;                               // barriers that count completed P V products
-constexpr int kThreads = 128 + kSplit * 128;             // producers + MMA issuers, then kSplit softmax warpgroups
+constexpr int kThreads = 128 + kSplit * 128 + 128;       // producers + MMA issuers, kSplit softmax warpgroups, V converters
+constexpr int kConvWarp0 = 4 + kSplit * 4;               // first warp of the converter warpgroup
 constexpr uint32_t kSubTileBytes = 128 * 128;            // [128 rows x 64 bf16], 16 KiB
 constexpr uint32_t kTileBytes = 2 * kSubTileBytes;       // 32 KiB: the Q tile, or a whole K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;          // 16 KiB: what one CTA holds of a K or V tile
 constexpr uint32_t kKSubBytes = 64 * 128;                // [64 keys x 64 channels] sub-tile of a K half
 constexpr uint32_t kSmemTiles = kTileBytes + (kRing + kRingV) * kHalfBytes;
-constexpr int kNumBars = 1 + 2 * kRing + 2 * kRingV + 2 * kSBuf + kPvRing + 1;
-constexpr uint32_t kBarBytes = 384;                      // barriers, TMEM slot, abort flag
-constexpr uint32_t kXchgBytes = 2 * kSplit * 128 * 4;    // [tile parity][column quarter][row] floats
+constexpr int kFRing = 4;                                // O correction factors in flight
+constexpr int kNumBars = 1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + 2 * kFRing + 1;
+constexpr uint32_t kBarBytes = 448;                      // barriers, TMEM slot, abort flag
+constexpr uint32_t kXchgBytes = (2 * kSplit + kFRing) * 128 * 4;   // row maxima [tile parity][column quarter][row], O factors [ring][row]
 constexpr uint32_t kSmemNeeded = kSmemTiles + kBarBytes + kXchgBytes;
 constexpr uint32_t kSmemBytes = 227 * 1024;              // everything an SM offers one CTA
 static_assert(8 * kNumBars + 16 <= kBarBytes, "barrier area too small");
@@ -125,12 +140,16 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   auto bar_sfull = [&](int b) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + b); };
   auto bar_pfull = [&](int b) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + kSBuf + b); };
   auto bar_pvdone = [&](int i) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + 2 * kSBuf + i); };
+  auto bar_vready = [&](int s) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + 2 * kSBuf + kPvRing + s); };
+  auto bar_f = [&](int i) { return bars + 8u * (1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + i); };
+  auto bar_corr = [&](int i) { return bars + 8u * (1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + kFRing + i); };
   const uint32_t bar_done = bars + 8u * (kNumBars - 1);
   unsigned char* base_generic = smem_raw + (base - raw);
   unsigned char* bars_generic = base_generic + kSmemTiles;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * kNumBars + 8);
   float* xchg = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [2][kSplit][128]
+  float* f_share = xchg + 2 * kSplit * 128;                            // [kFRing][128]
 
   const int h = blockIdx.x, mt = blockIdx.y, unit = blockIdx.z;      // the pair = heads (h & ~1, h | 1)
   const uint32_t rank = cluster_rank();                               // 0 = leader
@@ -143,9 +162,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   if (tid == 0) {
     mbar_init(bar_q, 1);
     for (int s = 0; s < kRing; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
-    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); }
+    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); mbar_init(bar_vready(s), 8); }
     for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 2 * kSplit * 4); }
     for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
+    for (int i = 0; i < kFRing; ++i) { mbar_init(bar_f(i), 4); mbar_init(bar_corr(i), 8); }
     mbar_init(bar_done, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -226,20 +246,25 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      // K halves complete on the leader's barrier (the leader posts both halves' bytes); a V half
+      // completes on its own CTA's barrier, where that CTA's softmax threads pick it up
       const uint32_t full_local = is_v ? bar_vfull(s) : bar_kfull(s);
-      const uint32_t full = leader_addr(full_local);
+      const uint32_t full = is_v ? full_local : leader_addr(full_local);
       const uint32_t sbase = ring + s * kHalfBytes;
-      if (leader && lane == 0) mbar_expect_tx(full_local, kTileBytes);
+      if (lane == 0) {
+        if (is_v) mbar_expect_tx(full_local, kHalfBytes);
+        else if (leader) mbar_expect_tx(full_local, kTileBytes);
+      }
       __syncwarp();
       if (j < past_tiles) {
         if (lane < 8) {
-          if (is_v) tma2_load_4d(sbase + lane * 2048u, tm_pages, full, int(rank) * 64, 0, g, page);
+          if (is_v) tma_load_4d(sbase + lane * 2048u, tm_pages, full, int(rank) * 64, 0, g, page);
           else tma2_load_4d(sbase + half * kKSubBytes + slot * 2048u, tm_pages, full, half * 64, 0, g, page);
         }
       } else {
         const int row0 = unit * nt + (j - past_tiles) * kBN;
         if (is_v) {
-          if (lane == 0) tma2_load_3d(sbase, tm_win, full, int(rank) * 64, g, row0);
+          if (lane == 0) tma_load_3d(sbase, tm_win, full, int(rank) * 64, g, row0);
         } else if (lane < 2) {
           tma2_load_3d(sbase + lane * kKSubBytes, tm_win, full, lane * 64, g, row0 + int(rank) * 64);
         }
@@ -251,12 +276,12 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     // copies complete on the leader's barriers, which only the leader can poll, so the peer waits
     // out the worst-case copy time instead
     if (!ok) {
-      if (leader) {
+      if (leader || is_v) {
         for (int j = max(0, issued - ring_n); j < issued; ++j) {
           const uint32_t fl = is_v ? bar_vfull(j % ring_n) : bar_kfull(j % ring_n);
           for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(fl, (j / ring_n) & 1); ++i) {}
         }
-        if (!is_v) for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
+        if (!is_v && leader) for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
       } else {
         __nanosleep(200000);
       }
@@ -296,24 +321,24 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           tc2_commit(bar_sfull(j % kSBuf));
         }
       } else {
-        constexpr uint32_t idesc_pv = make_idesc(true, 2 * kBM, kBN);
+        constexpr uint32_t idesc_pv = make_idesc_f16(true, 2 * kBM, kBN);
         const uint32_t tmem_o = tmem + kSBuf * 128;
         for (int i = 0; i < n_tiles && ok; ++i) {
           const int s = i % kRingV, b = i % kSBuf;
-          ok = mbar_wait(bar_vfull(s), (i / kRingV) & 1, abort_flag);
-          ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag);
+          // P(i) published by every softmax warp of both CTAs, which also turned V(i) into fp16
+          ok = mbar_wait(bar_vready(s), (i / kRingV) & 1, abort_flag);          // V(i) is fp16 in both CTAs
+          ok = ok && mbar_wait(bar_corr(i % kFRing), (i / kFRing) & 1, abort_flag);   // O is on P(i)'s maximum in both CTAs
+          ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag);      // P(i) published by both CTAs
           if (!ok) break;
           tc_fence_after();
           const uint32_t v_lo = desc_lo(v_ring + s * kHalfBytes, kSubTileBytes);
           const uint32_t p_tmem = tmem + b * 128;
 #pragma unroll
           for (int k = 0; k < kBN / 16; ++k) {
-            // 16 keys per step: B advances 16 rows of 128 bytes; A = 8 packed columns of the hi
-            // term, then the 8 columns of the lo term of the same keys against the same V rows.
+            // 16 keys per step: B advances 16 rows of 128 bytes, A 8 packed fp16 columns
             const uint32_t b_lo = v_lo + k * (2048u / 16u);
             const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
             mma2_ts(tmem_o, pa, b_lo, kHi, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
-            mma2_ts(tmem_o, pa + 16, b_lo, kHi, idesc_pv, 1u);
           }
           tc2_commit(bar_vempty(s));
           tc2_commit(bar_pvdone(i % kPvRing));
@@ -322,6 +347,60 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       }
     }
     __syncwarp();
+  } else if (warp >= kConvWarp0) {
+    // =========================== V converters ===========================
+    // This CTA's half of every V tile, as it landed (bf16), becomes fp16 in place, 128 bytes per
+    // thread; one arrival per warp on the leader's "V ready" barrier.
+    const int ct = tid - kConvWarp0 * 32;
+    const int q4 = warp & 3;                              // TMEM lane quadrant of this warp
+    const uint32_t o_row = tmem + (uint32_t(q4 * 32) << 16) + kSBuf * 128;
+    constexpr int kLag = 2;                               // V is converted this many tiles ahead of the correction
+    bool ok = true;
+    for (int it = 0; it < n_tiles + kLag && ok; ++it) {
+      if (it < n_tiles) {
+        const int vs = it % kRingV;
+        ok = mbar_wait(bar_vfull(vs), (it / kRingV) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint4* vp = reinterpret_cast<uint4*>(base_generic + (v_ring - base) + vs * kHalfBytes);
+        uint4 a[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) a[i] = vp[i * 128 + ct];      // consecutive threads, consecutive 16 bytes
+#pragma unroll
+        for (int i = 0; i < 8; ++i) vp[i * 128 + ct] = bf16x8_to_f16x8(a[i]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_addr(bar_vready(vs)));
+      }
+      const int j = it - kLag;
+      if (j >= 0) {
+        // The running maximum of tile j is known: where it grew, O (on the old maximum) is scaled
+        // down before P(j) V(j) is added.  The softmax threads do not wait for this.
+        ok = mbar_wait(bar_f(j % kFRing), (j / kFRing) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const float f = f_share[(j % kFRing) * 128 + ct];
+        if (__any_sync(0xffffffffu, f != 1.f)) {          // never for tile 0
+          // O must be quiescent: P V of every earlier tile complete
+          ok = mbar_wait(bar_pvdone((j - 1) % kPvRing), ((j - 1) / kPvRing) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t orr[32];
+            TMEM_LD32_WAIT(o_row + cc * 32, orr);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
+            TMEM_ST32(o_row + cc * 32, orr);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_addr(bar_corr(j % kFRing)));
+      }
+    }
   } else if (warp >= 4) {
     // =========================== softmax / epilogue ===========================
     // A query row (= TMEM lane) is shared by kSplit threads, 32 key columns each; the four warps
@@ -373,42 +452,31 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       if (!ok) break;                                     // the threads of a row leave together
       mx = fmaxf(fmaxf(xrow[0], xrow[128]), fmaxf(xrow[256], xrow[384]));
       const float m_new = fmaxf(m_used, mx * p.scale_log2);
-      const bool grow = m_new - m_used > kRescaleThreshold;     // also true for the first tile
-      if (j == 0) {
-        m_used = m_new;
-      } else if (__any_sync(0xffffffffu, grow)) {
-        // O must be quiescent: P V of every earlier tile complete (tile j's is not issued before
-        // this thread publishes P(j)).  One barrier per tile in a ring of 4, so the parity of the
-        // awaited phase cannot be confused with a later one.
-        ok = mbar_wait(bar_pvdone((j - 1) % kPvRing), ((j - 1) / kPvRing) & 1, abort_flag);
-        tc_fence_after();
-        const float f = grow ? ex2(m_used - m_new) : 1.f;
-        if (grow) { m_used = m_new; l *= f; }
-        uint32_t orr[32];
-        TMEM_LD32_WAIT(o_addr, orr);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * f);
-        TMEM_ST32(o_addr, orr);
+      const bool grow = m_new - m_used > kRescaleF16;           // also true for the first tile
+      // Where the maximum grew, O has to be scaled by f before P(j) V(j) is added: the correction
+      // warps do that, off this thread's path; tile 0 starts O, so its factor is 1.
+      const float f = grow ? ex2(m_used - m_new) : 1.f;         // 0 for the first tile (l = 0)
+      if (cq == 0) {
+        f_share[(j % kFRing) * 128 + row] = j > 0 ? f : 1.f;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_f(j % kFRing));
       }
-      // P = exp2(x - m) split into two bf16 terms (hi + lo): with outlier value channels a
-      // single bf16 P (8 significant bits) would cost up to |v| * 2^-9 of absolute error.
+      if (grow) { m_used = m_new; l *= f; }
+      // P = exp2(x - m) in fp16 (11 significant bits): with outlier value channels |v| ~ 40 a bf16
+      // P (8 bits) would cost up to |v| * 2^-9 = 0.08 of absolute error, fp16 at most |v| * 2^-12.
       const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm2 = pack2(-m_used, -m_used);
-      uint64_t sum_a = 0, sum_b = 0;                      // two (+0, +0) pairs
-      uint32_t pk[32];
+      // The row sum adds the values as rounded to fp16, the ones P V multiplies: numerator and
+      // denominator then carry the same rounding, which cancels where few keys dominate a row.
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+      uint32_t pk[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const uint64_t x = fma2(sv[i], scale2, negm2);
-        const float e0 = ex2(lo2(x)), e1 = ex2(hi2(x));
-        const uint64_t e = pack2(e0, e1);
-        if (i & 1) sum_b = add2(sum_b, e); else sum_a = add2(sum_a, e);
-        const uint32_t hi = pack_bf16(e0, e1);
-        pk[i] = hi;
-        const uint64_t lo = sub2(e, (uint64_t(hi & 0xFFFF0000u) << 32) | (hi << 16));
-        pk[16 + i] = pack_bf16(lo2(lo), hi2(lo));
+        pk[i] = pack_f16(ex2(lo2(x)), ex2(hi2(x)));
+        if (i & 1) add_f16x2(sum2, sum3, pk[i]); else add_f16x2(sum0, sum1, pk[i]);
       }
-      TMEM_ST32(s_addr, pk);
-      sum_a = add2(sum_a, sum_b);
-      l += lo2(sum_a) + hi2(sum_a);
+      TMEM_ST16(s_addr, pk);
+      l += (sum0 + sum1) + (sum2 + sum3);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();                                       // one arrival per warp: 32 of both CTAs' warps in all

@@ -174,6 +174,11 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       : "=l"(r[0]), "=l"(r[1]), "=l"(r[2]), "=l"(r[3]), "=l"(r[4]), "=l"(r[5]), "=l"(r[6]), "=l"(r[7]), "=l"(r[8]), "=l"(r[9]), "=l"(r[10]), "=l"(r[11]), "=l"(r[12]), "=l"(r[13]), "=l"(r[14]), "=l"(r[15]) \
       : "r"(taddr) \
       : "memory")
+#define TMEM_ST16(taddr, r) \
+  asm volatile( \
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" \
+      :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) \
+      : "memory")
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).
@@ -199,10 +204,37 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major, int m, int n)
   return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) |
          (uint32_t(m >> 4) << 24);
 }
+// The same with both operands in fp16 (format code 0 in the A and B fields).
+__host__ __device__ constexpr uint32_t make_idesc_f16(bool b_mn_major, int m, int n) {
+  return (1u << 4) | (uint32_t(b_mn_major) << 16) | (uint32_t(n >> 3) << 17) | (uint32_t(m >> 4) << 24);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// 8 bf16 values (16 bytes) to 8 fp16 values, exact for magnitudes in [2^-14, 65504].
+__device__ __forceinline__ uint4 bf16x8_to_f16x8(uint4 v) {
+  uint4 r;
+  r.x = pack_f16(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+  r.y = pack_f16(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+  r.z = pack_f16(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u));
+  r.w = pack_f16(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
+  return r;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -235,6 +267,12 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// (s0, s1) += the two fp16 halves of h2, added in fp32 (mixed-precision add, sm_100).
+__device__ __forceinline__ void add_f16x2(float& s0, float& s1, uint32_t h2) {
+  asm("{\n\t.reg .f16 a, b;\n\tmov.b32 {a, b}, %2;\n\tadd.rn.f32.f16 %0, a, %0;\n\tadd.rn.f32.f16 %1, b, %1;\n\t}"
+      : "+f"(s0), "+f"(s1) : "r"(h2));
+}
+
 // Barrier among the kWarps softmax warps that share a TMEM lane quadrant (hardware barrier
 // 1 + quadrant; barrier 0 is __syncthreads).  It also ANDs a predicate, so that all of them take
 // the same decision to go on or to give up.

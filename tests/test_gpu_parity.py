@@ -307,7 +307,12 @@ def test_tc_attention_repeatable_and_matches_general_kernel(B, monkeypatch, targ
         torch.cuda.synchronize()
         if ref is None:
             ref = outs[0].clone()
-            assert (gen - ref).abs().max().item() < 2e-3
+            # The single-CTA kernel rounds P to bf16 as a high and a low part (16 bits in all); the
+            # pair kernel rounds P to fp16 (relative error 2^-12), which the largest value channels
+            # of this workload (|v| up to about 40) turn into at most 40 * 2^-12 = 1e-2 absolute.
+            d = (gen - ref).abs()
+            assert d.max().item() < (1e-2 if kernel == "pair" else 2e-3)
+            assert d.mean().item() < 2e-4
         for o in outs:
             assert torch.equal(o, ref), f"run {rep}: tensor-core attention not repeatable"
     assert int(st.status.item()) == 0
