@@ -1,9 +1,9 @@
 // Step 6: cache append (Eq. 4) and representative keys of the blocks the step completes.
 //
 // One launch, two roles selected by blockIdx.x:
-//   copy CTAs   scatter the step's K / V rows into their pages (16-byte vectors);
-//   repr CTAs   one per (completed block, KV head, representative): each representative is the
-//               mean of B/r consecutive keys, read as 16-byte vectors by all threads at once
+//   copy CTAs   one per (page touched, K or V): the step's rows of that page, 16-byte vectors;
+//   repr CTAs   one warp per (completed block, KV head, representative): each representative is
+//               the mean of B/r consecutive keys, read as 16-byte vectors, eight in flight per lane,
 //               and accumulated in fp64 (exact for bf16 inputs, so the rounded table is
 //               bit-reproducible), rounded to the cache dtype; the inverse norm is taken from
 //               the rounded values in a fixed order.  Keys older than the step are
@@ -29,7 +29,7 @@ struct AppendParams {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
+__global__ void __launch_bounds__(kThreads, 3) append_kernel(AppendParams p) {
   const int unit = blockIdx.y;
   const int seq = unit / p.n_layers, layer_local = unit - seq * p.n_layers;
   const int64_t p0 = p.pos0[seq];
@@ -44,30 +44,49 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
   const int vpr = D / VN;
 
   if (int(blockIdx.x) < p.copy_ctas) {
-    // ---- copy role: one 16-byte vector of K and of V per thread iteration
-    const int64_t total = int64_t(p.n_tokens) * p.n_kv_heads * vpr;
-    for (int64_t idx = int64_t(blockIdx.x) * kThreads + tid; idx < total; idx += int64_t(p.copy_ctas) * kThreads) {
-      const int cv = int(idx % vpr);
-      const int g = int((idx / vpr) % p.n_kv_heads);
-      const int j = int(idx / (int64_t(vpr) * p.n_kv_heads));
-      const int64_t tok = p0 + j;
-      const int64_t lp = tok / p.page_tokens;
-      const int phys = lp < p.max_pages ? pt[lp] : -1;
-      if (phys < 0 || phys >= p.n_phys_pages) {
-        if (cv == 0) set_status(p.status, ACTQKV_DEV_BAD_PAGE);
-        continue;
+    // ---- copy role: one CTA per (page the step touches, K or V).  The page is contiguous in the
+    // cache, [head][token in page][D], and its tokens are contiguous in the window,
+    // [token][head][D]: thread-linear 16-byte vectors in the page's order, eight loads in flight
+    // per thread before the first store.
+    const int slot = int(blockIdx.x) >> 1;
+    const bool is_v = blockIdx.x & 1;
+    const int pt_tok = p.page_tokens;
+    const int64_t lp = p0 / pt_tok + slot;
+    const int64_t page0 = lp * pt_tok;
+    const int t_lo = int(max(p0, page0) - page0);
+    const int t_hi = int(min(p0 + p.n_tokens, page0 + pt_tok) - page0);
+    if (t_lo >= t_hi) return;
+    const int phys = lp < p.max_pages ? pt[lp] : -1;
+    if (phys < 0 || phys >= p.n_phys_pages) {
+      if (tid == 0) set_status(p.status, ACTQKV_DEV_BAD_PAGE);
+      return;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>((is_v ? vw : kw) + size_t(page0 - p0 + t_lo) * p.n_kv_heads * D);
+    uint4* dst = reinterpret_cast<uint4*>((is_v ? vp : kp) + size_t(phys) * page_elems);
+    // Thread = (row lane rl, channel vector cv); a row is one token of one head.  Heads in the
+    // unrolled loop, so that no index needs a division.
+    const int nt = t_hi - t_lo;                              // tokens of this page in the step
+    const int cv = tid % vpr, rl = tid / vpr, n_rl = kThreads / vpr;
+    constexpr int kUnroll = 8;
+    for (int t = rl; t < nt; t += n_rl) {
+      const uint4* s_row = src + size_t(t) * p.n_kv_heads * vpr + cv;
+      uint4* d_row = dst + size_t(t_lo + t) * vpr + cv;
+      for (int g0 = 0; g0 < p.n_kv_heads; g0 += kUnroll) {
+        uint4 val[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          if (g0 + u < p.n_kv_heads) val[u] = __ldg(s_row + (g0 + u) * vpr);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          if (g0 + u < p.n_kv_heads) d_row[size_t(g0 + u) * pt_tok * vpr] = val[u];
       }
-      const size_t src = (size_t(j) * p.n_kv_heads + g) * D + cv * VN;
-      const size_t dst = (size_t(phys) * p.n_kv_heads + g) * p.page_tokens * D +
-                         size_t(tok % p.page_tokens) * D + cv * VN;
-      *reinterpret_cast<uint4*>(kp + dst) = __ldg(reinterpret_cast<const uint4*>(kw + src));
-      *reinterpret_cast<uint4*>(vp + dst) = __ldg(reinterpret_cast<const uint4*>(vw + src));
     }
     return;
   }
 
-  // ---- repr role: one CTA per (completed block, KV head, representative)
-  const int rid = blockIdx.x - p.copy_ctas;
+  // ---- repr role: one warp per (completed block, KV head, representative)
+  const int warp = tid >> 5, lane = tid & 31;
+  const int rid = (int(blockIdx.x) - p.copy_ctas) * (kThreads / 32) + warp;
   const int i = rid % p.n_repr;
   const int g = (rid / p.n_repr) % p.n_kv_heads, nb = rid / (p.n_repr * p.n_kv_heads);
   const int64_t p1 = p0 + p.n_tokens;
@@ -76,68 +95,77 @@ __global__ void __launch_bounds__(kThreads) append_kernel(AppendParams p) {
   const int64_t b = done0 + nb;
   if (b >= done1) return;
   if (b >= p.n_cap) {
-    if (tid == 0) set_status(p.status, ACTQKV_DEV_TABLE_FULL);
+    if (lane == 0) set_status(p.status, ACTQKV_DEV_TABLE_FULL);
     return;
   }
-  // Thread t owns the 16-byte channel vector cv of rows rsub, rsub + rpp, ... of each chunk; the
-  // rpp partial sums of a channel are then added in a fixed order.  fp64 throughout: exact for
-  // bf16 keys, so the rounded table does not depend on the order.
-  extern __shared__ __align__(16) unsigned char append_smem[];
-  double* red = reinterpret_cast<double*>(append_smem);            // [rpp][D]
-  float* sq_s = reinterpret_cast<float*>(red + size_t(kThreads / vpr) * D);   // [D]
-  const int rpp = kThreads / vpr;                                   // rows per pass
-  const int cv = tid % vpr, rsub = tid / vpr;
+  // Lane = (row lane rsub, channel vector cv): it adds its vector of rows rsub, rsub + rpp, ... in
+  // fp64 (exact for bf16 keys, so the rounded table does not depend on the order), then the row
+  // lanes are added by shuffles in a fixed order.  vpr <= 32 lanes hold one row.
+  const int rpp = 32 / vpr;                                         // rows per pass of the warp
+  const int cv = lane % vpr, rsub = lane / vpr;
   const int seg = p.block / p.n_repr;
   const size_t row0 = ((size_t(unit) * p.n_kv_heads + g) * p.n_cap + size_t(b)) * p.n_repr;
   T* tab = static_cast<T*>(p.repr_k) + row0 * D;
   const int64_t blk0 = int64_t(p.n_init) + b * p.block;
-  {
-    const int lo = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? i * seg : i * seg + seg / 2;
-    const int hi = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? (i + 1) * seg : lo + 1;
-    double acc[VN];
+  const int lo = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? i * seg : i * seg + seg / 2;
+  const int hi = p.repr_mode == ACTQKV_REPR_CHUNK_MEAN ? (i + 1) * seg : lo + 1;
+  double acc[VN];
 #pragma unroll
-    for (int e = 0; e < VN; ++e) acc[e] = 0.0;
-    for (int r = lo + rsub; r < hi; r += rpp) {
-      const int64_t tok = blk0 + r;
-      const T* src = nullptr;
-      if (tok >= p0) {
-        src = kw + (size_t(tok - p0) * p.n_kv_heads + g) * D + cv * VN;
-      } else {
-        const int64_t lp = tok / p.page_tokens;
-        const int phys = lp < p.max_pages ? pt[lp] : -1;
-        if (phys < 0 || phys >= p.n_phys_pages) {
-          if (cv == 0) set_status(p.status, ACTQKV_DEV_BAD_PAGE);
+  for (int e = 0; e < VN; ++e) acc[e] = 0.0;
+  constexpr int kAhead = 8;                                         // 16-byte loads in flight per lane
+  for (int rb = lo + rsub; rb < hi; rb += rpp * kAhead) {
+    uint4 raw[kAhead];
+    bool have[kAhead];
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+      const int r = rb + u * rpp;
+      have[u] = false;
+      if (r < hi) {
+        const int64_t tok = blk0 + r;
+        const T* src = nullptr;
+        if (tok >= p0) {
+          src = kw + (size_t(tok - p0) * p.n_kv_heads + g) * D + cv * VN;
         } else {
-          src = kp + (size_t(phys) * p.n_kv_heads + g) * p.page_tokens * D + size_t(tok % p.page_tokens) * D + cv * VN;
+          const int64_t lp = tok / p.page_tokens;
+          const int phys = lp < p.max_pages ? pt[lp] : -1;
+          if (phys < 0 || phys >= p.n_phys_pages) {
+            if (cv == 0) set_status(p.status, ACTQKV_DEV_BAD_PAGE);
+          } else {
+            src = kp + (size_t(phys) * p.n_kv_heads + g) * p.page_tokens * D + size_t(tok % p.page_tokens) * D + cv * VN;
+          }
+        }
+        if (src) {
+          raw[u] = __ldg(reinterpret_cast<const uint4*>(src));
+          have[u] = true;
         }
       }
-      if (src) {
+    }
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u)
+      if (have[u]) {
         float kf[VN];
-        Vec16<T>::load_nc(src, kf);
+        Vec16<T>::unpack(raw[u], kf);
 #pragma unroll
         for (int e = 0; e < VN; ++e) acc[e] += double(kf[e]);
       }
-    }
-#pragma unroll
-    for (int e = 0; e < VN; ++e) red[size_t(rsub) * D + cv * VN + e] = acc[e];
-    __syncthreads();
-    if (tid < D) {
-      double t = 0.0;
-      for (int q = 0; q < rpp; ++q) t += red[size_t(q) * D + tid];
-      const double mean = t / double(hi - lo);
-      const T rounded = from_f32<T>(float(mean));   // fp64 -> fp32 -> dtype, both nearest-even
-      tab[size_t(i) * D + tid] = rounded;
-      const float stored = to_f32(rounded);
-      sq_s[tid] = stored * stored;
-    }
-    __syncthreads();
-    if (tid < 32) {                       // fixed order: lane partial sums, then a shuffle tree
-      float t = 0.f;
-      for (int cc = tid; cc < D; cc += 32) t += sq_s[cc];
-      t = warp_sum(t);
-      if (tid == 0) p.repr_inv_norm[row0 + i] = t > 0.f ? rsqrtf(t) : 0.f;
-    }
   }
+  // row lanes -> row lane 0, nearest partner first
+#pragma unroll
+  for (int e = 0; e < VN; ++e)
+    for (int o = vpr; o < 32; o <<= 1) acc[e] += __shfl_down_sync(0xffffffffu, acc[e], o);
+  float sq = 0.f;
+  if (rsub == 0) {
+    __align__(16) T outv[VN];
+#pragma unroll
+    for (int e = 0; e < VN; ++e) {
+      outv[e] = from_f32<T>(float(acc[e] / double(hi - lo)));          // fp64 -> fp32 -> dtype, both nearest-even
+      const float stored = to_f32(outv[e]);
+      sq = fmaf(stored, stored, sq);
+    }
+    *reinterpret_cast<uint4*>(tab + size_t(i) * D + cv * VN) = *reinterpret_cast<const uint4*>(outv);
+  }
+  sq = warp_sum(sq);                                                   // fixed order: per-lane sums, then a shuffle tree
+  if (lane == 0) p.repr_inv_norm[row0 + i] = sq > 0.f ? rsqrtf(sq) : 0.f;
 }
 
 }  // namespace
@@ -165,15 +193,13 @@ extern "C" int actqkv_append_window(const actqkv_config* cfg, const actqkv_batch
   p.max_pages = cfg->max_pages; p.n_phys_pages = cfg->n_phys_pages; p.n_layers = b.n_layers;
   p.repr_mode = cfg->repr_mode;
   const int vpr = cfg->head_dim * int(elt_size(cfg)) / 16;
-  const int64_t vecs = int64_t(n_tokens) * cfg->n_kv_heads * vpr;
-  p.copy_ctas = int(std::min<int64_t>((vecs + kThreads - 1) / kThreads, 296));
+  p.copy_ctas = 2 * (n_tokens / cfg->page_tokens + 2);      // K and V of every page the step can touch
   p.max_new_blocks = n_tokens / cfg->block + 2;
-  dim3 grid(p.copy_ctas + p.max_new_blocks * cfg->n_kv_heads * cfg->n_repr, b.units());
+  const int n_reprs = p.max_new_blocks * cfg->n_kv_heads * cfg->n_repr;
+  dim3 grid(p.copy_ctas + (n_reprs + kThreads / 32 - 1) / (kThreads / 32), b.units());
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  const size_t smem = sizeof(double) * size_t(kThreads / vpr) * cfg->head_dim + sizeof(float) * cfg->head_dim;
-  prefer_max_shared(append_kernel<__nv_bfloat16>);
-  prefer_max_shared(append_kernel<float>);
-  if (cfg->dtype == ACTQKV_BF16) append_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(p);
-  else append_kernel<float><<<grid, kThreads, smem, st>>>(p);
+  if (vpr > 32 || 32 % vpr != 0 || kThreads % vpr != 0) return ACTQKV_ERR_SHAPE;
+  if (cfg->dtype == ACTQKV_BF16) append_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(p);
+  else append_kernel<float><<<grid, kThreads, 0, st>>>(p);
   return launch_status();
 }
