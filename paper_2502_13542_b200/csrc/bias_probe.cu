@@ -2,9 +2,10 @@
 // probe-query (Eq. 9).
 //
 // The [n_tokens x D] query tile of one (unit, query head) is split by rows over S CTAs, and the
-// S x G CTAs of one KV head form a thread-block cluster (S * G <= 8).  Every CTA brings its rows from HBM into shared memory with one
-// bulk asynchronous copy per row (all in flight at once) and makes three passes over them with
-// 16-byte shared-memory loads:
+// S x G CTAs of one KV head form a thread-block cluster (S * G <= 8).  Every CTA brings its rows
+// from HBM into shared memory with tiled TMA loads of up to 256 rows each (the copy engine takes
+// about as long for a 256-byte request as for a 2 KiB one, so one request per row would cost more
+// than the data) and makes three passes over them with 16-byte shared-memory loads:
 //   1. per-channel sums of q and of (q - shift)^2, shift = the CTA's first row, which give
 //      the mean and the sum of squared deviations of its rows without a second pass; the row
 //      splits are merged pairwise (count, mean, M2) in a fixed order through distributed shared
@@ -14,7 +15,7 @@
 // Every reduction order is fixed, so results are bitwise reproducible.
 #include <cooperative_groups.h>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace cg = cooperative_groups;
 using namespace actqkv;
@@ -28,7 +29,7 @@ constexpr uint32_t kSpinLimit = 1u << 22;
 struct BiasProbeParams {
   const void* q;
   int n_tokens, n_q_heads, n_kv_heads, head_dim, group;
-  int split, rows_per_cta;
+  int split, rows_per_cta, box_rows, rows_alloc;   // rows_alloc: rows the tile holds (whole boxes)
   int64_t* stats_count;
   float* stats_mean;
   float* stats_m2;
@@ -48,7 +49,7 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) {
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams p) {   // 2 CTAs per SM on batched calls
+__global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
   constexpr int VN = Vec16<T>::N;             // elements per 16-byte vector
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams
   constexpr int PER = RL / NP;
   const int W = p.n_tokens, S = p.split, RP = p.rows_per_cta;
   T* tile = reinterpret_cast<T*>(smem_raw);
-  float* partial = reinterpret_cast<float*>(smem_raw + ((size_t(RP) * D * sizeof(T) + 127) & ~size_t(127)));   // [2][RL][D]
+  float* partial = reinterpret_cast<float*>(smem_raw + ((size_t(p.rows_alloc) * D * sizeof(T) + 127) & ~size_t(127)));   // [2][RL][D]
   float* level2 = partial + 2 * RL * D;       // [2][NP][D]
   // records read by other CTAs of the cluster (same offsets in every CTA)
   float* st_mean = level2 + 2 * NP * D;       // [D] mean of this CTA's rows
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams
 
   grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
   grid_launch_dependents();
-  // ---- 0. rows -> shared memory: one bulk copy per row, all in flight together
+  // ---- 0. rows -> shared memory
   constexpr uint32_t kRowBytes = D * sizeof(T);
   const uint32_t bar_addr = smem_addr(bar);
   if (tid == 0) {
@@ -92,13 +93,14 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  if (tid == 0 && nr > 0)
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(uint32_t(nr) * kRowBytes) : "memory");
-  __syncthreads();
-  for (int r = tid; r < nr; r += kThreads)
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(tile + size_t(r) * D)), "l"(qbase + size_t(r) * row_stride), "r"(kRowBytes), "r"(bar_addr)
-                 : "memory");
+  // q as [units * W rows][heads][D]: boxes of box_rows rows of this head.  Rows past the CTA's share
+  // (or past the tensor: zero fill) land in the tile's slack and are never read.
+  if (tid == 0 && nr > 0) {
+    const int n_box = (nr + p.box_rows - 1) / p.box_rows;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(uint32_t(n_box * p.box_rows) * kRowBytes) : "memory");
+    for (int bx = 0; bx < n_box; ++bx)
+      tc::tma_load_3d(smem_addr(tile + size_t(bx) * p.box_rows * D), &tm_q, bar_addr, 0, h, unit * W + r0 + bx * p.box_rows);
+  }
   // running statistics of this head, fetched while the copies fly
   const bool running = p.do_bias && p.stats_mode == ACTQKV_STATS_CUMULATIVE;
   float run_mean = 0.f, run_m2 = 0.f;
@@ -310,10 +312,372 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(BiasProbeParams
   cluster.sync();      // peers keep their shared memory alive until the leaders have read it
 }
 
+// The N / 2 packed fp32 pairs of a 16-byte vector (element 2i in the low half of pair i).
+template <typename T> struct Pairs;
+template <> struct Pairs<float> {
+  static constexpr int N2 = 2;
+  __device__ static __forceinline__ void get(const uint4& v, uint64_t (&out)[2]) {
+    asm("mov.b64 %0, {%1, %2};" : "=l"(out[0]) : "r"(v.x), "r"(v.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(out[1]) : "r"(v.z), "r"(v.w));
+  }
+};
+template <> struct Pairs<__nv_bfloat16> {
+  static constexpr int N2 = 4;
+  __device__ static __forceinline__ void get(const uint4& v, uint64_t (&out)[4]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) asm("mov.b64 %0, {%1, %2};" : "=l"(out[i]) : "r"(w[i] << 16), "r"(w[i] & 0xFFFF0000u));
+  }
+};
+
+// q viewed as [units * W rows][heads][D] with boxes of box_rows rows of one head.
+template <typename T, int D>
+bool encode_q(CUtensorMap* tm, const BiasProbeParams& p, int units, int box_rows) {
+  const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(p.n_q_heads), cuuint64_t(units) * cuuint64_t(p.n_tokens)};
+  const cuuint64_t strides[2] = {cuuint64_t(D) * sizeof(T), cuuint64_t(p.n_q_heads) * D * sizeof(T)};
+  const cuuint32_t box[3] = {cuuint32_t(D), 1u, cuuint32_t(box_rows)};
+  return tc::encode_plain(tm, sizeof(T) == 4, p.q, 3, dims, strides, box);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Batched calls (many (unit, head) items, e.g. all layers of a model in one launch): a persistent
+// kernel, one CTA per SM, no clusters.  A CTA takes whole items: the [n_tokens x D] tile of one
+// head arrives as up to kMaxChunks row chunks, one tiled TMA load and one barrier each; the column
+// sums of pass 1 are taken chunk by chunk while later chunks are still in flight; after the
+// statistics are merged a single second pass computes phi, the indicator a_j = ||phi_j||_1 and
+// sum_j a_j q_j together (the row is still in registers when its a_j is known), and hands every
+// chunk it has finished to the load of the CTA's NEXT item, so the loads never stop.  (A variant
+// in which every thread copied its own vectors with cp.async, without barriers, was slower: the
+// stage is bound by its instruction count, and the copies add to it.)  The KV-head probes (mean
+// over the G heads of a group, Eq. 9) are taken from the stored per-head probes by a small second
+// kernel.
+constexpr int kMaxChunks = 8;
+#ifndef STREAM_THREADS
+#define STREAM_THREADS 512
+#endif
+constexpr int kStreamThreads = STREAM_THREADS;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kStreamThreads, 1)
+bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams p, int n_items, int chunk_rows, int n_chunks) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  constexpr int VN = Vec16<T>::N;
+  constexpr int VPR = D / VN;
+  constexpr int RL = kStreamThreads / VPR;
+  constexpr int NP = kStreamThreads / D;
+  constexpr int NW = kStreamThreads / 32;     // warps
+  constexpr int PER = NW / NP;                // warps per second-level slice
+  constexpr int N2 = Pairs<T>::N2;
+  const int W = p.n_tokens;
+  const int rows_alloc = chunk_rows * n_chunks;
+  T* tile = reinterpret_cast<T*>(smem_raw);
+  float* partial = reinterpret_cast<float*>(smem_raw + ((size_t(rows_alloc) * D * sizeof(T) + 127) & ~size_t(127)));   // [2][NW][D]
+  float* level2 = partial + 2 * NW * D;       // [2][NP][D]
+  float* sum_a = level2 + 2 * NP * D;         // [D] first result of a column reduction
+  float* sum_b = sum_a + D;                   // [D] second result
+  float* mean_s = sum_b + D;                  // [D]
+  float* ivar_s = mean_s + D;                 // [D]
+  float* qsum_s = ivar_s + D;                 // [D] sum_j q_j of the item
+  float* red_s = qsum_s + D;                  // [32]
+  float* a_s = red_s + 32;                    // [W]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(a_s + ((W + 3) & ~3));   // [kMaxChunks]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cv = tid % VPR, rsub = tid / VPR;
+  const int passes_per_chunk = chunk_rows / RL;
+  const size_t row_stride = size_t(p.n_q_heads) * D;
+  constexpr uint32_t kRowBytes = D * sizeof(T);
+  const bool running = p.do_bias && p.stats_mode == ACTQKV_STATS_CUMULATIVE;
+
+  grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
+  grid_launch_dependents();
+  if (tid == 0) {
+    for (int c = 0; c < n_chunks; ++c) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bars + c)));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // Rows [c * chunk_rows, (c + 1) * chunk_rows) of an item -> shared memory (rows past n_tokens
+  // belong to the next unit or are zero fill; they are never read).  Every thread of the CTA has
+  // finished with the chunk's previous contents when this is called (a CTA barrier precedes it).
+  auto issue_chunk = [&](int item, int c) {
+    if (tid == 0) {
+      const int unit = item / p.n_q_heads, h = item - unit * p.n_q_heads;
+      const uint32_t bar = smem_addr(bars + c);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(uint32_t(chunk_rows) * kRowBytes) : "memory");
+      tc::tma_load_3d(smem_addr(tile + size_t(c) * chunk_rows * D), &tm_q, bar, 0, h, unit * W + c * chunk_rows);
+    }
+  };
+  auto wait_chunk = [&](int c, uint32_t parity) {
+    const uint32_t bar = smem_addr(bars + c);
+    bool landed = false;
+    for (uint32_t i = 0; i < kSpinLimit && !landed; ++i) {
+      uint32_t ok;
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                   : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      landed = ok != 0;
+    }
+    if (!landed && tid == 0) set_status(p.status, ACTQKV_DEV_TIMEOUT);     // goes on with whatever arrived
+  };
+  // dst0 / dst1 [D] = sums over the row lanes of a0 / a1, in a fixed order: the rows of a warp by
+  // shuffles, then the warps in two levels through shared memory (16-byte stores, no bank conflicts)
+  auto column_reduce2 = [&](float (&a0)[VN], float (&a1)[VN], float* dst0, float* dst1) {
+#pragma unroll
+    for (int o = VPR; o < 32; o <<= 1) {
+#pragma unroll
+      for (int e = 0; e < VN; ++e) {
+        a0[e] += __shfl_xor_sync(0xffffffffu, a0[e], o);
+        a1[e] += __shfl_xor_sync(0xffffffffu, a1[e], o);
+      }
+    }
+    __syncthreads();
+    if (lane < VPR) {
+#pragma unroll
+      for (int e = 0; e < VN; e += 4) {
+        *reinterpret_cast<float4*>(partial + warp * D + cv * VN + e) = make_float4(a0[e], a0[e + 1], a0[e + 2], a0[e + 3]);
+        *reinterpret_cast<float4*>(partial + NW * D + warp * D + cv * VN + e) = make_float4(a1[e], a1[e + 1], a1[e + 2], a1[e + 3]);
+      }
+    }
+    __syncthreads();
+    {
+      const int ch = tid % D, part = tid / D;
+      float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < PER; ++q) {
+        t0 += partial[(part * PER + q) * D + ch];
+        t1 += partial[NW * D + (part * PER + q) * D + ch];
+      }
+      level2[part * D + ch] = t0;
+      level2[NP * D + part * D + ch] = t1;
+    }
+    __syncthreads();
+    if (tid < D) {
+      float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < NP; ++q) { t0 += level2[q * D + tid]; t1 += level2[NP * D + q * D + tid]; }
+      dst0[tid] = t0;
+      dst1[tid] = t1;
+    }
+    __syncthreads();
+  };
+
+  if (int(blockIdx.x) < n_items)
+    for (int c = 0; c < n_chunks; ++c) issue_chunk(blockIdx.x, c);
+
+  uint32_t parity = 0;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x, parity ^= 1) {
+    const int unit = item / p.n_q_heads, h = item - unit * p.n_q_heads;
+    const size_t hd = (size_t(unit) * p.n_q_heads + h) * D;
+    const size_t uh = size_t(unit) * p.n_q_heads + h;
+    const int next = item + gridDim.x;
+    float run_mean = 0.f, run_m2 = 0.f;
+    int64_t run_count = 0;
+    if (running && tid < D) {
+      run_mean = p.stats_mean[hd + tid];
+      run_m2 = p.stats_m2[hd + tid];
+      run_count = p.stats_count[uh];
+    }
+    if (p.do_bias) {
+      // ---- pass 1, chunk by chunk as the rows land: sums of q and of (q - shift)^2, shift = row 0,
+      // on packed pairs of channels
+      uint64_t shift2[N2], s1p[N2], s2p[N2];
+#pragma unroll
+      for (int e = 0; e < N2; ++e) { s1p[e] = 0; s2p[e] = 0; shift2[e] = 0; }
+      for (int c = 0; c < n_chunks; ++c) {
+        wait_chunk(c, parity);
+        if (c == 0) Pairs<T>::get(*reinterpret_cast<const uint4*>(tile + cv * VN), shift2);
+        const T* src = tile + size_t(c * chunk_rows + rsub) * D + cv * VN;
+        const int n_here = min(passes_per_chunk, (W - c * chunk_rows - rsub + RL - 1) / RL);   // rows of this lane in the chunk
+#pragma unroll 2
+        for (int k = 0; k < n_here; ++k) {
+          uint64_t x[N2];
+          Pairs<T>::get(*reinterpret_cast<const uint4*>(src + size_t(k) * RL * D), x);
+#pragma unroll
+          for (int e = 0; e < N2; ++e) {
+            const uint64_t d = tc::sub2(x[e], shift2[e]);
+            s1p[e] = tc::add2(s1p[e], x[e]);
+            s2p[e] = tc::fma2(d, d, s2p[e]);
+          }
+        }
+      }
+      float s1[VN], s2[VN];
+#pragma unroll
+      for (int e = 0; e < N2; ++e) {
+        s1[2 * e] = tc::lo2(s1p[e]); s1[2 * e + 1] = tc::hi2(s1p[e]);
+        s2[2 * e] = tc::lo2(s2p[e]); s2[2 * e + 1] = tc::hi2(s2p[e]);
+      }
+      column_reduce2(s1, s2, sum_a, sum_b);
+      // ---- statistics of the window, merged into the running ones (Eq. 8)
+      if (tid < D) {
+        double n = double(W);
+        const double sh0 = double(to_f32(tile[tid]));
+        const double sq = double(sum_a[tid]), b2 = double(sum_b[tid]);
+        const double a = sq - n * sh0;             // sum (q - shift)
+        double mean = sq / n, m2 = fmax(b2 - a * a / n, 0.0);
+        qsum_s[tid] = sum_a[tid];
+        if (running) {
+          const double na = double(run_count), mean_a = double(run_mean), m2_a = double(run_m2);
+          const double nn = na + n, delta = mean - mean_a, w = n / nn;
+          mean = mean_a + delta * w;
+          m2 = m2_a + m2 + delta * delta * (na * w);
+          n = nn;
+          p.stats_mean[hd + tid] = float(mean);
+          p.stats_m2[hd + tid] = float(m2);
+          if (tid == 0) p.stats_count[uh] = run_count + W;
+        }
+        const double var = n > 1.0 ? m2 / (n - 1.0) : 0.0;
+        mean_s[tid] = float(mean);
+        ivar_s[tid] = float(1.0 / fmax(var, double(p.var_eps)));
+      }
+    } else {
+      for (int r = tid; r < W; r += kStreamThreads) a_s[r] = p.phi_l1[uh * W + r];
+    }
+    __syncthreads();
+    // ---- pass 2: phi, a_j = ||phi_j||_1 (Eq. 7) and this head's sum_j a_j q_j (and sum_j q_j when
+    // pass 1 did not run), on packed pairs of channels
+    uint64_t accp[N2], qsp[N2], mc2[N2], iv2[N2];
+#pragma unroll
+    for (int e = 0; e < N2; ++e) {
+      accp[e] = 0; qsp[e] = 0;
+      mc2[e] = p.do_bias ? tc::pack2(mean_s[cv * VN + 2 * e], mean_s[cv * VN + 2 * e + 1]) : 0;
+      iv2[e] = p.do_bias ? tc::pack2(ivar_s[cv * VN + 2 * e], ivar_s[cv * VN + 2 * e + 1]) : 0;
+    }
+    float a_tot = 0.f;
+    for (int c = 0; c < n_chunks; ++c) {
+      if (!p.do_bias) wait_chunk(c, parity);
+      const int r_base = c * chunk_rows + rsub;
+      const T* src = tile + size_t(r_base) * D + cv * VN;
+      // the row lanes of a warp run the same number of passes (a warp holds whole rows; W < r only
+      // switches the row off), so the shuffles below are convergent
+#pragma unroll 2
+      for (int k = 0; k < passes_per_chunk; ++k) {
+        const int r = r_base + k * RL;
+        const bool live = r < W;
+        uint64_t x[N2];
+        Pairs<T>::get(live ? *reinterpret_cast<const uint4*>(src + size_t(k) * RL * D) : make_uint4(0, 0, 0, 0), x);
+        float a;
+        if (p.do_bias) {
+          uint64_t part2 = 0;
+          if (p.phi_full && live) {
+            float* dst = p.phi_full + (size_t(unit) * W + r) * row_stride + size_t(h) * D + cv * VN;
+#pragma unroll
+            for (int e = 0; e < N2; ++e) {
+              const uint64_t d = tc::sub2(x[e], mc2[e]);
+              const uint64_t ph = tc::mul2(tc::mul2(d, d), iv2[e]);
+              *reinterpret_cast<float2*>(dst + 2 * e) = make_float2(tc::lo2(ph), tc::hi2(ph));
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < N2; ++e) {
+            const uint64_t d = tc::sub2(x[e], mc2[e]);
+            part2 = tc::fma2(tc::mul2(d, d), iv2[e], part2);
+          }
+          float part = live ? tc::lo2(part2) + tc::hi2(part2) : 0.f;
+#pragma unroll
+          for (int o = VPR >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+          a = part;                                // every lane of the row holds the same sum
+          if (live && cv == 0) a_s[r] = a;
+        } else {
+          a = live ? a_s[r] : 0.f;
+        }
+        if (cv == 0) a_tot += a;
+        if (p.do_probe) {
+          const uint64_t a2 = tc::pack2(a, a);
+#pragma unroll
+          for (int e = 0; e < N2; ++e) accp[e] = tc::fma2(a2, x[e], accp[e]);
+          if (!p.do_bias) {
+#pragma unroll
+            for (int e = 0; e < N2; ++e) qsp[e] = tc::add2(qsp[e], x[e]);
+          }
+        }
+      }
+      __syncthreads();                             // every thread is done with chunk c (and a_s has its rows)
+      if (next < n_items) issue_chunk(next, c);
+    }
+    float acc[VN], qs[VN];
+#pragma unroll
+    for (int e = 0; e < N2; ++e) {
+      acc[2 * e] = tc::lo2(accp[e]); acc[2 * e + 1] = tc::hi2(accp[e]);
+      qs[2 * e] = tc::lo2(qsp[e]); qs[2 * e + 1] = tc::hi2(qsp[e]);
+    }
+    if (p.do_bias && p.phi_l1)
+      for (int r = tid; r < W; r += kStreamThreads) p.phi_l1[uh * W + r] = a_s[r];
+    if (p.do_probe) {
+      // ---- Eq. 9 for this head
+      a_tot = warp_sum(a_tot);
+      if (lane == 0) red_s[warp] = a_tot;
+      column_reduce2(acc, qs, sum_a, sum_b);
+      if (tid < D) {
+        float t = 0.f;
+        for (int i = 0; i < kStreamThreads / 32; ++i) t += red_s[i];
+        const float qsum = p.do_bias ? qsum_s[tid] : sum_b[tid];
+        p.probe_qh[hd + tid] = t > 0.f ? sum_a[tid] / t : qsum / float(W);   // all-zero bias: uniform weights
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// KV-head probe = mean over the G query heads of the group (Eq. 9 under grouped-query attention).
+__global__ void probe_kv_kernel(const float* probe_qh, float* probe_kv, int n_q_heads, int n_kv_heads, int group, int D) {
+  const int unit = blockIdx.x / n_kv_heads, g = blockIdx.x - unit * n_kv_heads;
+  for (int ch = threadIdx.x; ch < D; ch += blockDim.x) {
+    float acc = 0.f;
+    for (int y = 0; y < group; ++y) acc += probe_qh[(size_t(unit) * n_q_heads + g * group + y) * D + ch];
+    probe_kv[(size_t(unit) * n_kv_heads + g) * D + ch] = acc / float(group);
+  }
+}
+
+// Returns 1 when the shape does not suit the streaming kernel (the caller takes the cluster kernel).
+template <typename T, int D>
+int launch_stream(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaStream_t st, int n_sm) {
+  constexpr int VN = Vec16<T>::N;
+  constexpr int RL = kStreamThreads / (D / VN), NP = kStreamThreads / D;
+  const int W = p.n_tokens;
+  const int per = std::max(1, (W + RL * kMaxChunks - 1) / (RL * kMaxChunks));
+  const int chunk_rows = RL * per, n_chunks = (W + chunk_rows - 1) / chunk_rows;
+  const size_t tile_bytes = (size_t(chunk_rows) * n_chunks * D * sizeof(T) + 127) & ~size_t(127);
+  const size_t smem = tile_bytes + sizeof(float) * (size_t(2) * (kStreamThreads / 32) * D + 2 * NP * D + 5 * D + 32 + ((W + 3) & ~3)) +
+                      8 * kMaxChunks;
+  if (smem > 227 * 1024) return 1;                    // the tile does not fit
+  if (chunk_rows > 256) return 1;                     // a box dimension holds at most 256
+  CUtensorMap tm_q;
+  if (!encode_q<T, D>(&tm_q, p, b.units(), chunk_rows)) return ACTQKV_ERR_LAUNCH;
+  auto kern = bias_probe_stream_kernel<T, D>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+    return ACTQKV_ERR_LAUNCH;
+  prefer_max_shared(kern);
+  const int n_items = b.units() * cfg->n_q_heads;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(std::min(n_items, n_sm), 1, 1);
+  lc.blockDim = dim3(kStreamThreads, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  allow_early_launch(attr[0]);
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  if (cudaLaunchKernelEx(&lc, kern, tm_q, p, n_items, chunk_rows, n_chunks) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ACTQKV_ERR_LAUNCH;
+  }
+  if (p.do_probe)
+    probe_kv_kernel<<<b.units() * cfg->n_kv_heads, D, 0, st>>>(p.probe_qh, p.probe_kv, cfg->n_q_heads, cfg->n_kv_heads,
+                                                                p.group, D);
+  return launch_status();
+}
+
 template <typename T, int D>
 int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaStream_t st) {
   const int W = p.n_tokens;
   const int cy = p.do_probe ? p.group : 1;
+  // Many items: the persistent streaming kernel (throughput); few: the cluster kernel (latency).
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (n_sm > 0 && b.units() * cfg->n_q_heads >= 2 * n_sm) {
+    const int rc = launch_stream<T, D>(cfg, b, p, st, n_sm);
+    if (rc <= 0) return rc;
+  }
   auto kern = bias_probe_kernel<T, D>;
   constexpr int VN = Vec16<T>::N;
   constexpr int RL = kThreads / (D / VN), NP = kThreads / D;
@@ -325,7 +689,11 @@ int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaS
     while (split > 1 && (W + split - 1) / split < 32) split >>= 1;
     p.split = split;
     p.rows_per_cta = (W + split - 1) / split;
-    const size_t tile_bytes = (size_t(p.rows_per_cta) * D * sizeof(T) + 127) & ~size_t(127);
+    p.box_rows = std::min(p.rows_per_cta, 256);                          // a box dimension holds at most 256
+    p.rows_alloc = (p.rows_per_cta + p.box_rows - 1) / p.box_rows * p.box_rows;
+    CUtensorMap tm_q;
+    if (!encode_q<T, D>(&tm_q, p, b.units(), p.box_rows)) return ACTQKV_ERR_LAUNCH;
+    const size_t tile_bytes = (size_t(p.rows_alloc) * D * sizeof(T) + 127) & ~size_t(127);
     const size_t smem = tile_bytes + sizeof(float) * (size_t(2) * RL * D + 2 * NP * D + 6 * D + 4 + 32 +
                                                        ((p.rows_per_cta + 3) & ~3)) + 16;
     if (smem > 220 * 1024) return ACTQKV_ERR_SHAPE;
@@ -345,7 +713,7 @@ int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaS
     allow_early_launch(attr[1]);
     lc.attrs = attr;
     lc.numAttrs = 2;
-    if (cudaLaunchKernelEx(&lc, kern, p) == cudaSuccess) return launch_status();
+    if (cudaLaunchKernelEx(&lc, kern, tm_q, p) == cudaSuccess) return launch_status();
     (void)cudaGetLastError();
   }
   return ACTQKV_ERR_LAUNCH;
