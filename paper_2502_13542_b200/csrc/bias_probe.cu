@@ -49,14 +49,13 @@ __device__ __forceinline__ uint32_t smem_addr(const void* p) {
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams p) {
+__global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   cg::cluster_group cluster = cg::this_cluster();
   constexpr int VN = Vec16<T>::N;             // elements per 16-byte vector
   constexpr int VPR = D / VN;                 // vectors per row
   constexpr int RL = kThreads / VPR;          // row lanes: thread (cv, rsub) owns vector cv of rows rsub + k * RL
   constexpr int NP = kThreads / D;            // second-level slices of the row lanes
-  constexpr int PER = RL / NP;
   const int W = p.n_tokens, S = p.split, RP = p.rows_per_cta;
   T* tile = reinterpret_cast<T*>(smem_raw);
   float* partial = reinterpret_cast<float*>(smem_raw + ((size_t(p.rows_alloc) * D * sizeof(T) + 127) & ~size_t(127)));   // [2][RL][D]
@@ -124,22 +123,34 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_co
   const int cv = tid % VPR, rsub = tid / VPR;
   const int n_pass = (nr + RL - 1) / RL;      // same trip count in every thread
   auto load_row = [&](int r, float (&f)[VN]) { Vec16<T>::load(tile + size_t(r) * D + cv * VN, f); };
-  // dst_k[D] = sum over the row lanes of acc_k, k < NA, in a fixed two-level order
-  auto column_reduce2 = [&](const float (&a0)[VN], const float (&a1)[VN], float* dst0, float* dst1) {
-    __syncthreads();
+  // dst0 / dst1 [D] = sums over the row lanes of a0 / a1, in a fixed order: the rows of a warp by
+  // shuffles, then the warps in two levels through shared memory (16-byte stores, no bank conflicts)
+  constexpr int NW = kThreads / 32, PERW = NW / NP;
+  auto column_reduce2 = [&](float (&a0)[VN], float (&a1)[VN], float* dst0, float* dst1) {
 #pragma unroll
-    for (int e = 0; e < VN; ++e) {
-      partial[rsub * D + cv * VN + e] = a0[e];
-      partial[RL * D + rsub * D + cv * VN + e] = a1[e];
+    for (int o = VPR; o < 32; o <<= 1) {
+#pragma unroll
+      for (int e = 0; e < VN; ++e) {
+        a0[e] += __shfl_xor_sync(0xffffffffu, a0[e], o);
+        a1[e] += __shfl_xor_sync(0xffffffffu, a1[e], o);
+      }
+    }
+    __syncthreads();
+    if (lane < VPR) {
+#pragma unroll
+      for (int e = 0; e < VN; e += 4) {
+        *reinterpret_cast<float4*>(partial + warp * D + cv * VN + e) = make_float4(a0[e], a0[e + 1], a0[e + 2], a0[e + 3]);
+        *reinterpret_cast<float4*>(partial + NW * D + warp * D + cv * VN + e) = make_float4(a1[e], a1[e + 1], a1[e + 2], a1[e + 3]);
+      }
     }
     __syncthreads();
     {
       const int ch = tid % D, part = tid / D;
       float t0 = 0.f, t1 = 0.f;
 #pragma unroll
-      for (int q = 0; q < PER; ++q) {
-        t0 += partial[(part * PER + q) * D + ch];
-        t1 += partial[RL * D + (part * PER + q) * D + ch];
+      for (int q = 0; q < PERW; ++q) {
+        t0 += partial[(part * PERW + q) * D + ch];
+        t1 += partial[NW * D + (part * PERW + q) * D + ch];
       }
       level2[part * D + ch] = t0;
       level2[NP * D + part * D + ch] = t1;
@@ -179,6 +190,9 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_co
     if (tid == 0) scal[1] = float(nr);
   }
 
+  float acc[VN];                       // this thread's share of sum_j a_j q_j
+#pragma unroll
+  for (int e = 0; e < VN; ++e) acc[e] = 0.f;
   if (p.do_bias) {
     cluster.sync();
     // ---- 2. merge the row splits, then the running statistics (Eq. 8 over all windows so far)
@@ -221,7 +235,8 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_co
       ivar_s[tid] = float(1.0 / fmax(var, double(p.var_eps)));
     }
     __syncthreads();
-    // ---- 3. phi and its L1 norm per token: the VPR lanes of a row add up by shuffles
+    // ---- 3. phi and its L1 norm a_j per token (the VPR lanes of a row add up by shuffles) and, with
+    // the row still in registers, its term of sum_j a_j q_j
     {
       float mc[VN], iv[VN];
 #pragma unroll
@@ -229,8 +244,11 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_co
       for (int k = 0; k < n_pass; ++k) {
         const int r = rsub + k * RL;
         float part = 0.f;
+        float f[VN];
+#pragma unroll
+        for (int e = 0; e < VN; ++e) f[e] = 0.f;
         if (r < nr) {
-          float f[VN], ph[VN];
+          float ph[VN];
           load_row(r, f);
 #pragma unroll
           for (int e = 0; e < VN; ++e) { const float d = f[e] - mc[e]; ph[e] = d * d * iv[e]; part += ph[e]; }
@@ -243,6 +261,10 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_co
 #pragma unroll
         for (int o = VPR >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
         if (r < nr && cv == 0) a_s[r] = part;
+        if (p.do_probe) {
+#pragma unroll
+          for (int e = 0; e < VN; ++e) acc[e] = fmaf(part, f[e], acc[e]);      // f = 0 for a row that is not there
+        }
       }
     }
     __syncthreads();
@@ -263,15 +285,17 @@ __global__ void __launch_bounds__(kThreads, 2) bias_probe_kernel(const __grid_co
     for (int r = tid; r < nr; r += kThreads) part += a_s[r];
     part = warp_sum(part);
     if (lane == 0) red_s[warp] = part;
-    float acc[VN], zero[VN];
+    float zero[VN];
 #pragma unroll
-    for (int e = 0; e < VN; ++e) { acc[e] = 0.f; zero[e] = 0.f; }
-    for (int r = rsub; r < nr; r += RL) {
-      float f[VN];
-      load_row(r, f);
-      const float w = a_s[r];
+    for (int e = 0; e < VN; ++e) zero[e] = 0.f;
+    if (!p.do_bias) {                    // the indicator was an input: the rows have not been passed yet
+      for (int r = rsub; r < nr; r += RL) {
+        float f[VN];
+        load_row(r, f);
+        const float w = a_s[r];
 #pragma unroll
-      for (int e = 0; e < VN; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+        for (int e = 0; e < VN; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+      }
     }
     column_reduce2(acc, zero, u_s, mean_s);      // mean_s is free by now: dummy destination
     if (tid == 0) {
