@@ -266,3 +266,49 @@ def test_decode_attention_splits_match_general_kernel(B, monkeypatch, n_new):
     with pytest.raises(B.ActQKVError):
         B.decode_attention(cfg, st.batch, q, k, v, n_new, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
                            st.sel_count, got, lse, n_splits=4, workspace=torch.zeros(64, device="cuda"))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", ["f32_d64", "bf16_d128"])
+def test_bias_probe_many_units_against_oracle(B, shape):
+    """Calls with at least two (unit, head) items per SM take the persistent streaming kernel
+    instead of the cluster kernel.  Two windows per unit (so the second merges into running
+    statistics, Eq. 8), the second one ragged (fewer tokens than a whole number of row chunks),
+    every unit with its own data, all outputs against the oracle (Eq. 7 - 9)."""
+    import torch
+    if shape == "f32_d64":
+        spec, U = wl.tiny_pr1(), 96              # 96 units x 4 heads
+    else:
+        spec, U = wl.llama3_8b_layer().replace(context=4096), 12    # 12 units x 32 heads
+    assert U * spec.n_q_heads >= 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    spec = spec.replace(n_layers=U)
+    cfg = B.make_config(spec)
+    batch = B.Batch(1, U, 0)
+    Hq, Hkv, D, W = spec.n_q_heads, spec.n_kv_heads, spec.head_dim, spec.window
+    f32 = dict(dtype=torch.float32, device="cuda")
+    count = torch.zeros(U, Hq, dtype=torch.int64, device="cuda")
+    mean, m2 = torch.zeros(U, Hq, D, **f32), torch.zeros(U, Hq, D, **f32)
+    probe_qh, probe_kv = torch.zeros(U, Hq, D, **f32), torch.zeros(U, Hkv, D, **f32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    runs = [orc.RunningStats(Hq, D) for _ in range(U)]
+    for t, n_tok in enumerate([W, W - 37]):
+        q_host = [wl.gen_q(spec, u, t)[:n_tok] for u in range(U)]
+        q = pu.to_device(np.stack(q_host), spec)
+        phi_l1 = torch.zeros(U, Hq, n_tok, **f32)
+        phi_full = torch.zeros(U, n_tok, Hq, D, **f32)
+        B.bias_probe(cfg, batch, q, n_tok, count, mean, m2, phi_l1, phi_full, probe_qh, probe_kv, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for u in range(U):
+            tag = f"{shape} unit {u} window {t}"
+            runs[u].update(q_host[u])
+            zbar, sigma2 = runs[u].mean, runs[u].variance()
+            phi, a = orc.activation_bias(q_host[u], zbar, sigma2)
+            pqh = orc.probe_query(q_host[u], a)
+            assert int(count[u, 0].item()) == runs[u].count
+            pu.assert_rel(pu.to_numpy(mean[u]), zbar, 1e-3 * np.abs(zbar).max() + 1e-30, tag + " mean")
+            pu.assert_rel(pu.to_numpy(m2[u]) / (runs[u].count - 1), sigma2, 1e-30, tag + " variance")
+            pu.assert_phi_like(pu.to_numpy(phi_l1[u]).T, a, tag + " phi_l1")
+            pu.assert_phi_like(pu.to_numpy(phi_full[u]), phi, tag + " phi")
+            pu.assert_probe(pu.to_numpy(probe_qh[u]), pqh, tag + " probe_qh")
+            pu.assert_probe(pu.to_numpy(probe_kv[u]), orc.kv_head_probe(pqh, Hkv), tag + " probe_kv")
