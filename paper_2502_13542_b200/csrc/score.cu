@@ -22,7 +22,7 @@ constexpr int kMaxPasses = 2;                       // row groups of one block h
 // its row's inverse norm and ONE shuffle tree over the warp finishes the block; the max
 // aggregation needs the r cosines separately and reduces row by row.
 template <typename T, int D, bool kMean>
-__global__ void __launch_bounds__(kScoreThreads)
+__global__ void __launch_bounds__(kScoreThreads, 2)
 score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
              const float* __restrict__ repr_inv_norm, const int32_t* __restrict__ n_cand,
              float* __restrict__ scores, int n_kv_heads, int r, int n_cap, int n_layers, int groups,
@@ -66,9 +66,26 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
       }
     }
   };
+  // Fast path (mean aggregation): a group of four blocks is 4 KiB of contiguous rows when
+  // r * D * sizeof(T) = 1 KiB per block: eight 512-byte warp loads at fixed offsets from one base,
+  // the sixteen inverse norms by one load and shuffles.  Whole groups only; a ragged last group
+  // takes the general loads.
+  constexpr int kVec = 8;                                // 512-byte vectors per group
+  struct Raw { uint4 v[kVec]; float nrm; };
+  const bool fast_shape = kMean && size_t(r) * D * sizeof(T) == 1024;
+  auto load_fast = [&](int bg, Raw& x) {
+    const uint4* pch = reinterpret_cast<const uint4*>(repr_k + (head_rows + size_t(bg) * r) * D) + lane;
+#pragma unroll
+    for (int u = 0; u < kVec; ++u) x.v[u] = __ldg(pch + u * 32);
+    x.nrm = lane < kBlocksPerWarp * r ? __ldg(inv + size_t(bg) * r + lane) : 0.f;
+  };
+  auto full = [&](int gi) { return gi < groups && b0 + (gi + 1) * kBlocksPerWarp <= n; };
+  auto exists = [&](int gi) { return gi < groups && b0 + gi * kBlocksPerWarp < n; };
   // the first group's loads go out before anything else, then the probe
   Group ga, gb;
-  load_group(b0, ga);
+  Raw ra, rb;
+  const bool first_fast = fast_shape && full(0);
+  if (first_fast) load_fast(b0, ra); else load_group(b0, ga);
   grid_dependency_wait();            // the table is older than the stream's previous kernel; the probe is not
   grid_launch_dependents();
   const float* pg = probe_kv + (size_t(unit) * n_kv_heads + g) * D;
@@ -145,6 +162,56 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
       }
     }
   };
+  if constexpr (kMean) if (fast_shape) {
+    // the four block sums of a group are reduced together (6 shuffles instead of 20): halves swap
+    // block pairs, quarters swap blocks, then three steps inside each quarter
+    auto score_fast = [&](int bg, const Raw& x) {
+      float accb[kBlocksPerWarp];
+#pragma unroll
+      for (int bi = 0; bi < kBlocksPerWarp; ++bi) {
+        accb[bi] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {                    // the block's two vectors
+          const int u = 2 * bi + k;
+          float row[VN];
+          Vec16<T>::unpack(x.v[u], row);
+          float dot = 0.f;
+#pragma unroll
+          for (int e = 0; e < VN; ++e) dot = fmaf(pv[e], row[e], dot);
+          const float w = __shfl_sync(0xffffffffu, x.nrm, u * RPP + sub);   // row u * RPP + sub of the group
+          accb[bi] = fmaf(dot, w, accb[bi]);
+        }
+      }
+      const bool up16 = lane & 16, up8 = lane & 8;
+      const float t0 = __shfl_xor_sync(0xffffffffu, up16 ? accb[0] : accb[2], 16);
+      const float t1 = __shfl_xor_sync(0xffffffffu, up16 ? accb[1] : accb[3], 16);
+      const float k0 = (up16 ? accb[2] : accb[0]) + t0, k1 = (up16 ? accb[3] : accb[1]) + t1;
+      float k = (up8 ? k1 : k0) + __shfl_xor_sync(0xffffffffu, up8 ? k0 : k1, 8);
+      k += __shfl_xor_sync(0xffffffffu, k, 4);
+      k += __shfl_xor_sync(0xffffffffu, k, 2);
+      k += __shfl_xor_sync(0xffffffffu, k, 1);
+      if ((lane & 7) == 0) out[bg + 2 * (lane >> 4) + ((lane >> 3) & 1)] = k * inv_pn / float(r);
+    };
+    auto ragged = [&](int gi) {                            // a last, partly filled group: general loads
+      const int bg = b0 + gi * kBlocksPerWarp;
+      load_group(bg, ga);
+      score_group(bg, ga);
+    };
+    if (!first_fast) { score_group(b0, ga); return; }      // b0 + 4 > n: the only group of this warp
+    // invariant at the loop head: if group gi is whole, ra holds it
+    for (int gi = 0; exists(gi);) {
+      if (!full(gi)) { ragged(gi); break; }
+      if (full(gi + 1)) load_fast(b0 + (gi + 1) * kBlocksPerWarp, rb);
+      score_fast(b0 + gi * kBlocksPerWarp, ra);
+      ++gi;
+      if (!exists(gi)) break;
+      if (!full(gi)) { ragged(gi); break; }
+      if (full(gi + 1)) load_fast(b0 + (gi + 1) * kBlocksPerWarp, ra);
+      score_fast(b0 + gi * kBlocksPerWarp, rb);
+      ++gi;
+    }
+    return;
+  }
   // double-buffered: the next group's loads are in flight while the current group is scored
   for (int gi = 0; gi < groups; gi += 2) {
     const int bg = b0 + gi * kBlocksPerWarp;
