@@ -375,7 +375,10 @@ bool encode_q(CUtensorMap* tm, const BiasProbeParams& p, int units, int box_rows
 // stage is bound by its instruction count, and the copies add to it.)  The KV-head probes (mean
 // over the G heads of a group, Eq. 9) are taken from the stored per-head probes by a small second
 // kernel.
-constexpr int kMaxChunks = 8;
+#ifndef MAX_CHUNKS
+#define MAX_CHUNKS 2
+#endif
+constexpr int kMaxChunks = MAX_CHUNKS;
 #ifndef STREAM_THREADS
 #define STREAM_THREADS 512
 #endif
@@ -573,8 +576,49 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
       const T* src = tile + size_t(r_base) * D + cv * VN;
       // the row lanes of a warp run the same number of passes (a warp holds whole rows; W < r only
       // switches the row off), so the shuffles below are convergent
+      int k_done = 0;
+      if (p.do_bias && p.do_probe && !p.phi_full && VPR >= 4) {
+        // four rows at a time: their four sums over the VPR lanes of a row are reduced together
+        // (halves swap row pairs, quarters swap rows: 3 + log2(VPR / 4) shuffles instead of
+        // 4 log2(VPR)) and handed back to every lane of the row by four more
+        for (; k_done + 4 <= passes_per_chunk; k_done += 4) {
+          uint64_t x[4][N2];
+          float part[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const bool live = r_base + (k_done + j) * RL < W;
+            Pairs<T>::get(live ? *reinterpret_cast<const uint4*>(src + size_t(k_done + j) * RL * D) : make_uint4(0, 0, 0, 0), x[j]);
+            uint64_t part2 = 0;
+#pragma unroll
+            for (int e = 0; e < N2; ++e) {
+              const uint64_t d = tc::sub2(x[j][e], mc2[e]);
+              part2 = tc::fma2(tc::mul2(d, d), iv2[e], part2);
+            }
+            part[j] = live ? tc::lo2(part2) + tc::hi2(part2) : 0.f;
+          }
+          constexpr int H1 = VPR / 2, H2 = VPR / 4;
+          const bool up1 = lane & H1, up2 = lane & H2;
+          const float t0 = __shfl_xor_sync(0xffffffffu, up1 ? part[0] : part[2], H1);
+          const float t1 = __shfl_xor_sync(0xffffffffu, up1 ? part[1] : part[3], H1);
+          const float k0 = (up1 ? part[2] : part[0]) + t0, k1 = (up1 ? part[3] : part[1]) + t1;
+          float kv = (up2 ? k1 : k0) + __shfl_xor_sync(0xffffffffu, up2 ? k0 : k1, H2);
+#pragma unroll
+          for (int o = H2 >> 1; o > 0; o >>= 1) kv += __shfl_xor_sync(0xffffffffu, kv, o);
+          const int row_lane0 = lane & ~(VPR - 1);           // first lane of this row's lane group
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float a = __shfl_sync(0xffffffffu, kv, row_lane0 + (j >> 1) * H1 + (j & 1) * H2);
+            const int r = r_base + (k_done + j) * RL;
+            if (r < W && cv == 0) a_s[r] = a;
+            if (cv == 0) a_tot += a;
+            const uint64_t a2 = tc::pack2(a, a);
+#pragma unroll
+            for (int e = 0; e < N2; ++e) accp[e] = tc::fma2(a2, x[j][e], accp[e]);
+          }
+        }
+      }
 #pragma unroll 2
-      for (int k = 0; k < passes_per_chunk; ++k) {
+      for (int k = k_done; k < passes_per_chunk; ++k) {
         const int r = r_base + k * RL;
         const bool live = r < W;
         uint64_t x[N2];
