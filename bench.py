@@ -161,7 +161,8 @@ def build_states(spec, n_copies, device):
     for t in range(T - 1):
         q = pu.to_device(wl.gen_q(spec, 0, t)[None], spec, device)
         k, v = wl.gen_kv(spec, 0, t)
-        base.step(q, pu.to_device(k[None], spec, device), pu.to_device(v[None], spec, device), out)
+        k, v = pu.to_device(k[None], spec, device), pu.to_device(v[None], spec, device)
+        base.step(q, k, v, out)
     torch.cuda.synchronize()
     q = pu.to_device(wl.gen_q(spec, 0, T - 1)[None], spec, device)
     k, v = wl.gen_kv(spec, 0, T - 1)
@@ -557,10 +558,18 @@ def run_decode16(args):
         B.score_select(cfg, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, st.budget_state, st.scores,
                        st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
 
+    ws = None
+    if args.decode_splits > 1:           # split form of the decode kernel, with a caller-owned workspace
+        ws = torch.zeros(B.decode_workspace_bytes(cfg, states[0].batch, 1, args.decode_splits), dtype=torch.uint8, device=dev)
+
     def attention():
         st = cur()
-        B.retrieval_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
-                              st.sel_count, out, None, st.status)
+        if ws is None:
+            B.retrieval_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                                  st.sel_count, out, None, st.status)
+        else:
+            B.decode_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                               st.sel_count, out, None, args.decode_splits, ws, st.status)
         it["i"] += 1
     e = 2
     n_blocks = [wl.n_candidates(spec, int(c)) for c in ctx]
@@ -606,6 +615,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="layer32k", choices=["layer32k", "stack32", "decode16"],
                     help="layer32k = the headline line; the others print per-stage HBM figures on batched shapes")
+    ap.add_argument("--decode-splits", type=int, default=1,
+                    help="decode16 workload: key-stream splits per (sequence, KV head) of the decode attention")
     ap.add_argument("--profile-region", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
