@@ -257,7 +257,18 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const uint32_t o_addr = tmem + lane_addr + kSBuf * 128 + b * 64;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
+    // A warp whose 32 rows hold no query (single-token decode fills G rows of the tile) only keeps
+    // the barrier phases in step: nothing is read from its rows of P or O, and the exponentials,
+    // issue slots and TMEM traffic it would spend go to the warps that have rows.
+    const bool warp_used = q4 * 32 < nt * G;
+    if (!warp_used) {
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int sb = j % kSBuf;
+        ok = mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
+        mbar_arrive(bar_pfull(sb));
+      }
+    }
+    for (int j = 0; warp_used && j < n_tiles; ++j) {
       const int sb = j % kSBuf;
       ok = ok && mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
       tc_fence_after();
@@ -345,10 +356,12 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       mbar_arrive(bar_pfull(sb));
     }
     // ---- epilogue: the row sum over both column halves, then this thread's 64 channels of O / l
-    ok = ok && mbar_wait(bar_done, 0, abort_flag);
+    ok = ok && warp_used && mbar_wait(bar_done, 0, abort_flag);
     float* xrow = xchg + (n_tiles & 1) * 256 + row;
-    xrow[b * 128] = l;
-    ok = pair_sync_and(q4, ok);
+    if (warp_used) {
+      xrow[b * 128] = l;
+      ok = pair_sync_and(q4, ok);
+    }
     if (ok) {
       tc_fence_after();
       const float lsum = l + xrow[(1 - b) * 128];
