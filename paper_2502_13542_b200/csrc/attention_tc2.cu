@@ -12,17 +12,18 @@
 // 32 KiB per tile instead of 64, and the rings hold 6 K halves and 5 V halves.  No TMA multicast
 // is used: each CTA fetches its own halves.
 //
-// Roles per CTA (768 threads): warp 0 K producer, warp 2 V producer, warps 1 and 3 the MMA issuers
-// (leader CTA = cluster rank 0 only; warp 1: S = Q K^T, warp 3: O += P V), warps 4-19 softmax with
-// FOUR threads per query row (32 key columns each; the four warps of a TMEM lane quadrant share a
-// scheduler, which hides their latencies), warps 20-23 V conversion and O correction.
+// Roles per CTA (512 threads): warp 0 K producer, warp 2 V producer, warps 1 and 3 the MMA issuers
+// (leader CTA = cluster rank 0 only; warp 1: S = Q K^T, warp 3: O += P V), warps 4-11 softmax: each
+// owns 16 query rows (TMEM lanes) and reads all 128 key columns of their S rows with one 16x256b
+// load, so a row's maximum and sum are finished by shuffles inside a quad of threads and no softmax
+// warp waits for another one inside a tile; warps 12-15 V conversion and O correction.
 //
 // P is kept in fp16 (11 significant bits; one tcgen05.mma per 16 keys, half the tensor-pipe time of
-// a bf16 high + low pair), so V must be fp16 too (kind::f16 wants both operands alike): warps 20-23
+// a bf16 high + low pair), so V must be fp16 too (kind::f16 wants both operands alike): warps 12-15
 // convert each CTA's half of a V tile in place after it landed, two tiles ahead of its use.  The row
 // sum adds the fp16-rounded P, so numerator and denominator carry the same rounding.  fp16 tops out
 // at 65504, so the running maximum used for P may lag the true one by at most 2^8; when it has to
-// move, O is rescaled by warps 20-23 between two P V products, off the softmax threads' path.
+// move, O is rescaled by warps 12-15 between two P V products, off the softmax threads' path.
 // Cross-CTA signalling:
 //   K loads of both CTAs complete on the LEADER's "full" barriers (cta_group::2 form of the load);
 //   V loads complete on the loading CTA's barrier; its converter warps then arrive on the leader's
@@ -45,11 +46,11 @@ constexpr int kRing = 6;                                 // K halves in flight
 constexpr int kRingV = 5;                                // V halves in flight
 // fp16 P: exp2(x - m) must stay below 65504, so the running maximum may lag by at most 2^8
 constexpr float kRescaleF16 = 8.0f;
-constexpr int kSplit = 4;                                // softmax threads per query row (32 key columns each)
+constexpr int kSoftmaxWarps = 8;                         // each owns 16 query rows (TMEM lanes) and all 128 key columns of a tile
 constexpr int kSBuf = 3;                                 // S/P buffers in TMEM
 constexpr int kPvRing = 4;                               // barriers that count completed P V products
-constexpr int kThreads = 128 + kSplit * 128 + 128;       // producers + MMA issuers, kSplit softmax warpgroups, V converters
-constexpr int kConvWarp0 = 4 + kSplit * 4;               // first warp of the converter warpgroup
+constexpr int kThreads = 128 + kSoftmaxWarps * 32 + 128; // producers + MMA issuers, softmax warps, V converters / O correction
+constexpr int kConvWarp0 = 4 + kSoftmaxWarps;            // first warp of the converter warpgroup
 constexpr uint32_t kSubTileBytes = 128 * 128;            // [128 rows x 64 bf16], 16 KiB
 constexpr uint32_t kTileBytes = 2 * kSubTileBytes;       // 32 KiB: the Q tile, or a whole K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;          // 16 KiB: what one CTA holds of a K or V tile
@@ -58,7 +59,7 @@ constexpr uint32_t kSmemTiles = kTileBytes + (kRing + kRingV) * kHalfBytes;
 constexpr int kFRing = 4;                                // O correction factors in flight
 constexpr int kNumBars = 1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + 2 * kFRing + 1;
 constexpr uint32_t kBarBytes = 448;                      // barriers, TMEM slot, abort flag
-constexpr uint32_t kXchgBytes = (2 * kSplit + kFRing) * 128 * 4;   // row maxima [tile parity][column quarter][row], O factors [ring][row]
+constexpr uint32_t kXchgBytes = (2 + kFRing) * 128 * 4;  // final row sums and maxima [row], O factors [ring][row]
 constexpr uint32_t kSmemNeeded = kSmemTiles + kBarBytes + kXchgBytes;
 constexpr uint32_t kSmemBytes = 227 * 1024;              // everything an SM offers one CTA
 static_assert(8 * kNumBars + 16 <= kBarBytes, "barrier area too small");
@@ -148,8 +149,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   unsigned char* bars_generic = base_generic + kSmemTiles;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * kNumBars + 8);
-  float* xchg = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [2][kSplit][128]
-  float* f_share = xchg + 2 * kSplit * 128;                            // [kFRing][128]
+  float* l_share = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [128] row sums, for the epilogue
+  float* m_share = l_share + 128;                                        // [128] running maxima, for the log-sum-exp
+  float* f_share = m_share + 128;                                        // [kFRing][128] O correction factors
 
   const int h = blockIdx.x, mt = blockIdx.y, unit = blockIdx.z;      // the pair = heads (h & ~1, h | 1)
   const uint32_t rank = cluster_rank();                               // 0 = leader
@@ -163,9 +165,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     mbar_init(bar_q, 1);
     for (int s = 0; s < kRing; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
     for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); mbar_init(bar_vready(s), 8); }
-    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 2 * kSplit * 4); }
+    for (int b = 0; b < kSBuf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pfull(b), 2 * kSoftmaxWarps); }
     for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
-    for (int i = 0; i < kFRing; ++i) { mbar_init(bar_f(i), 4); mbar_init(bar_corr(i), 8); }
+    for (int i = 0; i < kFRing; ++i) { mbar_init(bar_f(i), kSoftmaxWarps); mbar_init(bar_corr(i), 8); }
     mbar_init(bar_done, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -337,7 +339,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           for (int k = 0; k < kBN / 16; ++k) {
             // 16 keys per step: B advances 16 rows of 128 bytes, A 8 packed fp16 columns
             const uint32_t b_lo = v_lo + k * (2048u / 16u);
-            const uint32_t pa = p_tmem + (k >> 1) * 32 + (k & 1) * 8;
+            const uint32_t pa = p_tmem + k * 8;
             mma2_ts(tmem_o, pa, b_lo, kHi, idesc_pv, (i > 0 || k > 0) ? 1u : 0u);
           }
           tc2_commit(bar_vempty(s));
@@ -403,122 +405,153 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
   } else if (warp >= 4) {
     // =========================== softmax / epilogue ===========================
-    // A query row (= TMEM lane) is shared by kSplit threads, 32 key columns each; the four warps
-    // of a lane quadrant sit on the same scheduler, so their stalls overlap.
-    const int cq = (warp >> 2) - 1;                       // column quarter of every tile
-    const int q4 = warp & 3;                              // TMEM lane quadrant of this warp
-    const int row = q4 * 32 + lane;                       // query row inside the tile
-    const uint32_t lane_addr = uint32_t(q4 * 32) << 16;
-    const uint32_t o_addr = tmem + lane_addr + kSBuf * 128 + cq * 32;
-    float m_used = -INFINITY, l = 0.f;
+    // A warp owns 16 query rows (TMEM lanes) and reads all 128 key columns of their S rows with ONE
+    // 16x256b load: the four threads of a quad share two rows (lane g and g + 8; thread q of the
+    // quad holds columns 8k + 2q, 8k + 2q + 1 of both, k = 0..15).  A row's maximum and sum are
+    // finished by two shuffles inside the quad, so no warp ever waits for another one inside a
+    // tile, and the eight softmax warps drift apart: while one is bound by the special-function
+    // unit (exponentials) another reads TMEM and takes maxima.  The packed fp16 pair of columns
+    // (8k + 2q, +1) is P column 4k + q: exactly the register layout of the 16x128b store.
+    const int sw = warp - 4;
+    const int q4 = sw & 3, hw = sw >> 2;                  // TMEM lane quadrant (= warp % 4); lower / upper 16 lanes
+    const int qd = lane & 3, g8 = lane >> 2;
+    const int row0 = q4 * 32 + hw * 16 + g8, row1 = row0 + 8;      // this thread's two query rows inside the tile
+    const uint32_t lane16 = uint32_t(q4 * 32 + hw * 16) << 16;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;     // running maxima (log2 units) and partial row sums
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
       const int sb = j % kSBuf;
-      ok = ok && mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
+      ok = mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
-      const uint32_t s_addr = tmem + lane_addr + sb * 128 + cq * 32;
-      uint64_t sv[16];
-      TMEM_LD32P_WAIT(s_addr, sv);
-      // key-validity limit: ragged last past tile, or the causal diagonal of the last tile
-      int limit = kBN;
-      if (j < past_tiles) limit = min(kBN, n_past - j * kBN);
-      else if (j == n_tiles - 1) limit = row + 1;
-      limit -= cq * 32;                                   // in this thread's column numbering
+      const uint32_t s_addr = tmem + lane16 + sb * 128;
+      uint64_t sv[32];                                    // sv[2k] row0, sv[2k + 1] row1
+      TMEM_LD16X256P_WAIT(s_addr, sv);
+      // key-validity limits: ragged last past tile, or the causal diagonal of the last tile
+      int lim0 = kBN, lim1 = kBN;
+      if (j < past_tiles) lim0 = lim1 = min(kBN, n_past - j * kBN);
+      else if (j == n_tiles - 1) { lim0 = row0 + 1; lim1 = row1 + 1; }
       const bool masked = (j == n_tiles - 1) || (j == past_tiles - 1 && (n_past % kBN) != 0);   // CTA-uniform
-      float mx = -INFINITY, mx2 = -INFINITY;
+      float mx0 = -INFINITY, mx1 = -INFINITY;
       if (masked) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float x0 = 2 * i < limit ? lo2(sv[i]) : -INFINITY;
-          const float x1 = 2 * i + 1 < limit ? hi2(sv[i]) : -INFINITY;
-          sv[i] = pack2(x0, x1);
-          mx = max3(mx, x0, x1);
+        for (int k = 0; k < 16; ++k) {
+          const int col = 8 * k + 2 * qd;
+          const float a0 = col < lim0 ? lo2(sv[2 * k]) : -INFINITY, a1 = col + 1 < lim0 ? hi2(sv[2 * k]) : -INFINITY;
+          const float b0 = col < lim1 ? lo2(sv[2 * k + 1]) : -INFINITY, b1 = col + 1 < lim1 ? hi2(sv[2 * k + 1]) : -INFINITY;
+          sv[2 * k] = pack2(a0, a1);
+          sv[2 * k + 1] = pack2(b0, b1);
+          mx0 = max3(mx0, a0, a1);
+          mx1 = max3(mx1, b0, b1);
         }
       } else {
-        float mx3 = -INFINITY, mx4 = -INFINITY;           // four independent chains
+        float mx0b = -INFINITY, mx1b = -INFINITY;         // two chains per row
 #pragma unroll
-        for (int i = 0; i < 16; i += 4) {
-          mx = max3(mx, lo2(sv[i]), hi2(sv[i]));
-          mx2 = max3(mx2, lo2(sv[i + 1]), hi2(sv[i + 1]));
-          mx3 = max3(mx3, lo2(sv[i + 2]), hi2(sv[i + 2]));
-          mx4 = max3(mx4, lo2(sv[i + 3]), hi2(sv[i + 3]));
+        for (int k = 0; k < 16; k += 2) {
+          mx0 = max3(mx0, lo2(sv[2 * k]), hi2(sv[2 * k]));
+          mx1 = max3(mx1, lo2(sv[2 * k + 1]), hi2(sv[2 * k + 1]));
+          mx0b = max3(mx0b, lo2(sv[2 * k + 2]), hi2(sv[2 * k + 2]));
+          mx1b = max3(mx1b, lo2(sv[2 * k + 3]), hi2(sv[2 * k + 3]));
         }
-        mx = fmaxf(max3(mx, mx2, mx3), mx4);
+        mx0 = fmaxf(mx0, mx0b);
+        mx1 = fmaxf(mx1, mx1b);
       }
-      // the row's maximum over the four column quarters
-      float* xrow = xchg + (j & 1) * (kSplit * 128) + row;
-      xrow[cq * 128] = mx;
-      ok = quadrant_sync_and<kSplit>(q4, ok);
-      if (!ok) break;                                     // the threads of a row leave together
-      mx = fmaxf(fmaxf(xrow[0], xrow[128]), fmaxf(xrow[256], xrow[384]));
-      const float m_new = fmaxf(m_used, mx * p.scale_log2);
-      const bool grow = m_new - m_used > kRescaleF16;           // also true for the first tile
+      // the rows' maxima over the quad
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float n0 = fmaxf(m0, mx0 * p.scale_log2), n1 = fmaxf(m1, mx1 * p.scale_log2);
+      const bool grow0 = n0 - m0 > kRescaleF16, grow1 = n1 - m1 > kRescaleF16;   // also true for the first tile
       // Where the maximum grew, O has to be scaled by f before P(j) V(j) is added: the correction
       // warps do that, off this thread's path; tile 0 starts O, so its factor is 1.
-      const float f = grow ? ex2(m_used - m_new) : 1.f;         // 0 for the first tile (l = 0)
-      if (cq == 0) {
-        f_share[(j % kFRing) * 128 + row] = j > 0 ? f : 1.f;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_f(j % kFRing));
+      const float f0 = grow0 ? ex2(m0 - n0) : 1.f, f1 = grow1 ? ex2(m1 - n1) : 1.f;   // 0 for the first tile (l = 0)
+      if (qd == 0) {
+        f_share[(j % kFRing) * 128 + row0] = j > 0 ? f0 : 1.f;
+        f_share[(j % kFRing) * 128 + row1] = j > 0 ? f1 : 1.f;
       }
-      if (grow) { m_used = m_new; l *= f; }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_f(j % kFRing));
+      if (grow0) { m0 = n0; l0 *= f0; }
+      if (grow1) { m1 = n1; l1 *= f1; }
       // P = exp2(x - m) in fp16 (11 significant bits): with outlier value channels |v| ~ 40 a bf16
       // P (8 bits) would cost up to |v| * 2^-9 = 0.08 of absolute error, fp16 at most |v| * 2^-12.
-      const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm2 = pack2(-m_used, -m_used);
-      // The row sum adds the values as rounded to fp16, the ones P V multiplies: numerator and
-      // denominator then carry the same rounding, which cancels where few keys dominate a row.
-      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-      uint32_t pk[16];
+      // The row sum adds the values as rounded to fp16, the ones P V multiplies.  P overwrites the
+      // first 64 columns of these rows of S, all of which this warp already holds.
+      const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2);
+      const uint64_t negm0 = pack2(-m0, -m0), negm1 = pack2(-m1, -m1);
+      float s0a = 0.f, s0b = 0.f, s1a = 0.f, s1b = 0.f;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const uint64_t x = fma2(sv[i], scale2, negm2);
-        pk[i] = pack_f16(ex2(lo2(x)), ex2(hi2(x)));
-        if (i & 1) add_f16x2(sum2, sum3, pk[i]); else add_f16x2(sum0, sum1, pk[i]);
+      for (int hh = 0; hh < 2; ++hh) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const int k = 8 * hh + kk;
+          const uint64_t x0 = fma2(sv[2 * k], scale2, negm0), x1 = fma2(sv[2 * k + 1], scale2, negm1);
+          pk[2 * kk] = pack_f16(ex2(lo2(x0)), ex2(hi2(x0)));
+          pk[2 * kk + 1] = pack_f16(ex2(lo2(x1)), ex2(hi2(x1)));
+          add_f16x2(s0a, s0b, pk[2 * kk]);
+          add_f16x2(s1a, s1b, pk[2 * kk + 1]);
+        }
+        TMEM_ST16X128_X8(s_addr + hh * 32, pk);
       }
-      TMEM_ST16(s_addr, pk);
-      l += (sum0 + sum1) + (sum2 + sum3);
+      l0 += s0a + s0b;
+      l1 += s1a + s1b;
       tmem_wait_st();
       tc_fence_before();
-      __syncwarp();                                       // one arrival per warp: 32 of both CTAs' warps in all
+      __syncwarp();                                       // one arrival per warp: 16 of both CTAs' warps in all
       if (lane == 0) mbar_arrive_cluster(leader_addr(bar_pfull(sb)));
     }
-    // ---- epilogue: the row sum over the four column quarters, then this thread's 32 channels of O / l
+    // ---- epilogue: the rows' sums over the quad, handed over in shared memory; then thread = row,
+    // warp hw takes channels [64 hw, 64 hw + 64) of O / l
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    if (qd == 0) {
+      l_share[row0] = l0; l_share[row1] = l1;
+      m_share[row0] = m0; m_share[row1] = m1;
+    }
     ok = ok && mbar_wait(bar_done, 0, abort_flag);
-    float* xrow = xchg + (n_tiles & 1) * (kSplit * 128) + row;
-    xrow[cq * 128] = l;
-    ok = quadrant_sync_and<kSplit>(q4, ok);
+    ok = pair_sync_and(q4, ok);                           // the two warps of a lane quadrant
     if (ok) {
       tc_fence_after();
-      const float lsum = (xrow[0] + xrow[128]) + (xrow[256] + xrow[384]);
+      const int row = q4 * 32 + lane;
+      const float lsum = l_share[row];
       const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
       const size_t tok = size_t(unit) * nt + size_t(mt) * kBM + row;
-      const int col = cq * 32;
-      uint32_t orr[32];
-      TMEM_LD32_WAIT(o_addr, orr);
-      if (p.out_bf16) {
-        __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
+      const uint32_t o_row = tmem + (uint32_t(q4 * 32) << 16) + kSBuf * 128;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 v;
-          v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
-          v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
-          v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
-          v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
-          *reinterpret_cast<uint4*>(ob + 8 * i) = v;
-        }
-      } else {
-        float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
+      for (int cc = 0; cc < 2; ++cc) {
+        const int col = hw * 64 + cc * 32;
+        uint32_t orr[32];
+        TMEM_LD32_WAIT(o_row + col, orr);
+        if (p.out_bf16) {
+          __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float4 v;
-          v.x = __uint_as_float(orr[4 * i + 0]) * inv; v.y = __uint_as_float(orr[4 * i + 1]) * inv;
-          v.z = __uint_as_float(orr[4 * i + 2]) * inv; v.w = __uint_as_float(orr[4 * i + 3]) * inv;
-          *reinterpret_cast<float4*>(of + 4 * i) = v;
+          for (int i = 0; i < 4; ++i) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(orr[8 * i + 0]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+            *reinterpret_cast<uint4*>(ob + 8 * i) = v;
+          }
+        } else {
+          float* of = static_cast<float*>(p.a.out) + (tok * p.n_q_heads + h) * kD + col;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float4 v;
+            v.x = __uint_as_float(orr[4 * i + 0]) * inv; v.y = __uint_as_float(orr[4 * i + 1]) * inv;
+            v.z = __uint_as_float(orr[4 * i + 2]) * inv; v.w = __uint_as_float(orr[4 * i + 3]) * inv;
+            *reinterpret_cast<float4*>(of + 4 * i) = v;
+          }
         }
       }
-      if (p.a.lse && cq == 0)
+      if (p.a.lse && hw == 0)
         p.a.lse[(size_t(unit) * p.n_q_heads + h) * nt + size_t(mt) * kBM + row] =
-            (m_used + log2f(lsum)) * 0.6931471805599453f;
+            (m_share[row] + log2f(lsum)) * 0.6931471805599453f;
     }
   }
 
