@@ -90,7 +90,7 @@ class ClockSampler(threading.Thread):
 # DRAM traffic of one launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
 # ncu capture of this workload), valid only for the kernel source it was taken on: the figure is
 # reported while the sha256 of the kernel file still starts with the recorded digits, else null.
-ATTENTION_TRAFFIC = {"source_sha256_16": "48b80b8b6bebcc76", "bytes_per_launch": 23661312}
+ATTENTION_TRAFFIC = {"source_sha256_16": "8f25a2402d12373f", "bytes_per_launch": 23673856}
 
 
 def attention_traffic():
