@@ -296,9 +296,19 @@ def test_bias_probe_many_units_against_oracle(B, shape):
         q = pu.to_device(np.stack(q_host), spec)
         phi_l1 = torch.zeros(U, Hq, n_tok, **f32)
         phi_full = torch.zeros(U, n_tok, Hq, D, **f32)
+        # the two-call form (Eq. 7-8, then Eq. 9) on copies of the statistics: same kernels, other switches
+        count2, mean2, m22 = count.clone(), mean.clone(), m2.clone()
+        phi_l1_b, pqh_b, pkv_b = torch.zeros_like(phi_l1), torch.zeros_like(probe_qh), torch.zeros_like(probe_kv)
+        B.activation_bias(cfg, batch, q, n_tok, count2, mean2, m22, phi_l1_b, None, status)
+        B.probe_query(cfg, batch, q, n_tok, phi_l1_b, pqh_b, pkv_b, status)
         B.bias_probe(cfg, batch, q, n_tok, count, mean, m2, phi_l1, phi_full, probe_qh, probe_kv, status)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
+        assert torch.equal(count2, count) and torch.equal(mean2, mean) and torch.equal(m22, m2)
+        assert torch.equal(phi_l1_b, phi_l1)
+        for got, want, nm in ((pqh_b, probe_qh, "probe_qh"), (pkv_b, probe_kv, "probe_kv")):
+            for u in range(U):
+                pu.assert_probe(pu.to_numpy(got[u]), pu.to_numpy(want[u]).astype(np.float64), f"{shape} unit {u} two-call {nm}")
         for u in range(U):
             tag = f"{shape} unit {u} window {t}"
             runs[u].update(q_host[u])
