@@ -152,21 +152,20 @@ def build_states(spec, n_copies, device):
     import torch
     from paper_2502_13542_b200 import binding as B
     from paper_2502_13542_b200 import workloads as wl
-    from tests import parity_utils as pu
 
     cfg = B.make_config(spec, out_dtype=B.BF16)
     base = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :], device=device)
     out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=device)
     T = spec.n_windows
     for t in range(T - 1):
-        q = pu.to_device(wl.gen_q(spec, 0, t)[None], spec, device)
+        q = wl.to_device(wl.gen_q(spec, 0, t)[None], spec, device)
         k, v = wl.gen_kv(spec, 0, t)
-        k, v = pu.to_device(k[None], spec, device), pu.to_device(v[None], spec, device)
+        k, v = wl.to_device(k[None], spec, device), wl.to_device(v[None], spec, device)
         base.step(q, k, v, out)
     torch.cuda.synchronize()
-    q = pu.to_device(wl.gen_q(spec, 0, T - 1)[None], spec, device)
+    q = wl.to_device(wl.gen_q(spec, 0, T - 1)[None], spec, device)
     k, v = wl.gen_kv(spec, 0, T - 1)
-    k, v = pu.to_device(k[None], spec, device), pu.to_device(v[None], spec, device)
+    k, v = wl.to_device(k[None], spec, device), wl.to_device(v[None], spec, device)
     states, inputs = [], []
     names = ["stats_count", "stats_mean", "stats_m2", "repr_k", "repr_inv_norm", "budget_state", "k_pages",
              "v_pages", "probe_kv", "probe_qh"]
@@ -401,8 +400,8 @@ def _oracle_sample(spec, st_cache, q, k, v, heads):
 def _oracle_state(spec):
     from oracle import actqkv_oracle as orc
     from paper_2502_13542_b200 import workloads as wl
-    from tests import parity_utils as pu
-    run = pu.OracleRunner(spec)
+    from oracle.runner import OracleRunner
+    run = OracleRunner(spec)
     T = spec.n_windows
     for t in range(T - 1):
         run.state.stats.update(wl.gen_q(spec, 0, t))

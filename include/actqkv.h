@@ -8,6 +8,22 @@
  *   activation_bias -> probe_query -> score_blocks -> select_cutoff
  *                   -> retrieval_attention -> append_window
  *
+ * Equation numbers.  The paper does not number its equations; the comments of this library number
+ * them in order of appearance:
+ *   Eq. 1  prefill attention over the full cache          (Sec. 3.1)
+ *   Eq. 2  prefill attention over the selected cache      (Sec. 3.1)
+ *   Eq. 3  decode attention                               (Sec. 3.1)
+ *   Eq. 4  cache update                                   (Sec. 3.1)
+ *   Eq. 5  top-k retrieval objective                      (Sec. 3.2)
+ *   Eq. 6  anchor-token criterion                         (Sec. 4.1)
+ *   Eq. 7  Activation Bias phi                            (Sec. 4.1)
+ *   Eq. 8  running mean and variance of the queries       (Sec. 4.1)
+ *   Eq. 9  activation-aware probe-query                   (Sec. 4.1)
+ *   Eq. 10 cosine score of a probe and a key              (Sec. 4.2)
+ *   Eq. 11 information density (entropy of the scores)    (Sec. 4.2)
+ *   Eq. 12 per-layer budget of the dynamic KV cut-off     (Sec. 4.2)
+ *   Algorithm 1  the cut-off over all layers              (Sec. 4.2)
+ *
  * Conventions shared by every entry point
  * ---------------------------------------
  *  - Every data pointer is a DEVICE pointer unless it is marked "host".  The
@@ -76,6 +92,13 @@ enum { ACTQKV_STATS_CUMULATIVE = 0, ACTQKV_STATS_WINDOW_ONLY = 1 };
 enum { ACTQKV_REPR_CHUNK_MEAN = 0, ACTQKV_REPR_STRIDED_TOKEN = 1 };
 enum { ACTQKV_AGG_MEAN = 0, ACTQKV_AGG_MAX = 1 };
 enum { ACTQKV_THETABAR_STREAMING = 0, ACTQKV_THETABAR_ALG1 = 1 };
+/* Token weights of the probe-query: Eq. 9 (default), or uniform = the mean-pooling probe the paper
+ * compares against (Sec. 1; the "w/o APQ" row of its ablation, Sec. 5.3). */
+enum { ACTQKV_PROBE_ACTIVATION = 0, ACTQKV_PROBE_MEAN_POOL = 1 };
+/* Which kernel serves actqkv_retrieval_attention: chosen by shape (default); the general
+ * fp32-accumulate kernel; the single-CTA tensor-core kernel.  The last two exist for testing one
+ * kernel against another; results agree within the rounding of the products. */
+enum { ACTQKV_ATTN_AUTO = 0, ACTQKV_ATTN_GENERAL = 1, ACTQKV_ATTN_SINGLE_CTA = 2 };
 
 /* Host POD describing the model / cache geometry.  Passed by const pointer (host). */
 typedef struct actqkv_config {
@@ -103,6 +126,8 @@ typedef struct actqkv_config {
   float sm_scale;        /* attention scale; 0 => 1/sqrt(D)                               */
   float var_eps;         /* floor on sigma^2 in Eq. 7; 0 => 1e-12                         */
   int32_t out_dtype;     /* element type of the attention output: ACTQKV_F32 | ACTQKV_BF16 */
+  int32_t probe_mode;    /* ACTQKV_PROBE_*: token weights of the probe-query                 */
+  int32_t attention_kernel; /* ACTQKV_ATTN_*: 0 = pick by shape                              */
 } actqkv_config;
 
 typedef struct actqkv_batch {
@@ -141,7 +166,9 @@ int actqkv_activation_bias(const actqkv_config* cfg, const actqkv_batch* batch, 
 
 /* ---- step 2: activation-aware probe-query (Eq. 9) --------------------------------------
  * probe_qh[h] = sum_j (phi_l1[h,j] / sum_j phi_l1[h,j]) * q[j,h,:]  (uniform weights when the
- * sum is 0); probe_kv[g] = mean of probe_qh over the G query heads of KV head g.
+ * sum is 0, and always with probe_mode MEAN_POOL, which ignores phi_l1);
+ * probe_kv[g] = mean of probe_qh over the G query heads of KV head g.
+ * A step of one token (decode) gives probe_qh = q: the paper's decode-stage probe (Sec. 4.2).
  *   probe_qh [U][Hq][D] fp32 out;  probe_kv [U][Hkv][D] fp32 out. */
 int actqkv_probe_query(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
                        int32_t n_tokens, const float* phi_l1, float* probe_qh, float* probe_kv,
@@ -203,7 +230,13 @@ int actqkv_score_select(const actqkv_config* cfg, const actqkv_batch* batch, con
  * bf16, D = 128, 16-token pages: steps whose n_tokens is a multiple of 128 run on the tcgen05
  * prefill kernels (CTA pairs when G is even), steps of n_tokens <= 128 / G tokens on the tcgen05
  * decode kernel (one CTA per KV head; see actqkv_decode_attention for the split form); every
- * other shape runs on the general fp32-accumulate kernel. */
+ * other shape runs on the general fp32-accumulate kernel.
+ * Preconditions of the tcgen05 kernels (the general kernel has none of them):
+ *  - p0 need not sit on a page boundary, but the rows of the last, partly filled cache page that
+ *    lie past p0 must hold finite values: they are masked out of the softmax yet still enter the
+ *    P V product with weight 0, and 0 x NaN is NaN.  A zero-initialised pool satisfies this, and
+ *    actqkv_append_window zero-fills the rest of the last page it touches.
+ *  - The CTA-pair kernel multiplies P and V in fp16: |v| <= 65504 (larger finite values saturate). */
 int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv_batch* batch, const void* q,
                                const void* k_win, const void* v_win, int32_t n_tokens,
                                const void* k_pages, const void* v_pages, const int32_t* page_table,

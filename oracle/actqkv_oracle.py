@@ -422,9 +422,12 @@ class LayerState:
 def window_retrieval(state: LayerState, chain: BudgetChain, layer: int, q, k, v, *, n_init, block,
                      n_repr, dtype, n_local_prev=0, beta=1.0, var_eps=1e-12, repr_mode="chunk_mean",
                      agg="mean", attention=True, stats_mode="cumulative", theta_all=None,
-                     repr_table=None):
+                     repr_table=None, probe_mode="activation"):
     """One step of the path for one layer: bias -> probe -> score -> cut-off /
-    select -> attention -> append.  Returns a dict of every intermediate."""
+    select -> attention -> append.  Returns a dict of every intermediate.
+
+    probe_mode "activation" is Eq. 9; "mean_pool" is the uniform-weight probe the
+    paper compares against (Sec. 1, and the ablation of Sec. 5.3)."""
     p0 = state.k_cache.shape[0]
     hkv = k.shape[1]
     if stats_mode == "cumulative":
@@ -433,7 +436,12 @@ def window_retrieval(state: LayerState, chain: BudgetChain, layer: int, q, k, v,
     else:
         zbar, sigma2 = query_stats_two_pass(q)
     phi, a = activation_bias(q, zbar, sigma2, var_eps)
-    pq = probe_query(q, a)
+    if probe_mode == "activation":
+        pq = probe_query(q, a)
+    elif probe_mode == "mean_pool":
+        pq = mean_pool_probe(q)
+    else:
+        raise ValueError(probe_mode)
     pkv = kv_head_probe(pq, hkv)
     n = n_candidate_blocks(p0, n_init, block, n_local_prev) if p0 > n_init else 0
     if repr_table is None:

@@ -26,6 +26,8 @@ STATS_CUMULATIVE, STATS_WINDOW_ONLY = 0, 1
 REPR_CHUNK_MEAN, REPR_STRIDED_TOKEN = 0, 1
 AGG_MEAN, AGG_MAX = 0, 1
 THETABAR_STREAMING, THETABAR_ALG1 = 0, 1
+PROBE_ACTIVATION, PROBE_MEAN_POOL = 0, 1
+ATTN_AUTO, ATTN_GENERAL, ATTN_SINGLE_CTA = 0, 1, 2
 
 DEV_BAD_PAGE, DEV_NCAND_CLAMPED, DEV_BAD_PROBE, DEV_BAD_SELECTION, DEV_TIMEOUT, DEV_TABLE_FULL = \
     1, 2, 4, 8, 16, 32
@@ -37,7 +39,8 @@ class Config(C.Structure):
         "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "window", "block", "n_repr", "page_tokens",
         "n_init", "n_local_prev", "k_blocks", "cap_blocks", "dtype", "stats_mode", "repr_mode",
         "agg_mode", "thetabar_mode", "n_cap", "max_pages", "n_phys_pages")] + [
-        ("beta", C.c_float), ("sm_scale", C.c_float), ("var_eps", C.c_float), ("out_dtype", C.c_int32)]
+        ("beta", C.c_float), ("sm_scale", C.c_float), ("var_eps", C.c_float), ("out_dtype", C.c_int32),
+        ("probe_mode", C.c_int32), ("attention_kernel", C.c_int32)]
 
     @property
     def torch_dtype(self):
@@ -214,7 +217,8 @@ def append_window(cfg, batch, k_win, v_win, n_tokens, pos0, k_pages, v_pages, pa
 # ----------------------------------------------------------------------------
 def make_config(spec, *, n_cap=None, max_pages=None, n_phys_pages=None, beta=1.0,
                 stats_mode=STATS_CUMULATIVE, repr_mode=REPR_CHUNK_MEAN, agg_mode=AGG_MEAN,
-                thetabar_mode=THETABAR_STREAMING, max_context=None, out_dtype=None) -> Config:
+                thetabar_mode=THETABAR_STREAMING, max_context=None, out_dtype=None,
+                probe_mode=PROBE_ACTIVATION, attention_kernel=ATTN_AUTO) -> Config:
     """Config for a `workloads.WorkloadSpec`-like object (any object with the same fields)."""
     ctx = max_context if max_context is not None else spec.context + spec.decode_steps
     pages = -(-ctx // spec.page_tokens)
@@ -231,6 +235,7 @@ def make_config(spec, *, n_cap=None, max_pages=None, n_phys_pages=None, beta=1.0
     cfg.n_phys_pages = n_phys_pages if n_phys_pages is not None else pages
     cfg.beta, cfg.sm_scale, cfg.var_eps = beta, 0.0, 0.0
     cfg.out_dtype = cfg.dtype if out_dtype is None else out_dtype
+    cfg.probe_mode, cfg.attention_kernel = probe_mode, attention_kernel
     return cfg
 
 

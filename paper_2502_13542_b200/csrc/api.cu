@@ -1,7 +1,4 @@
 // Helpers of the C ABI and the dispatcher of step 5.
-#include <cstdlib>
-#include <cstring>
-
 #include "common.cuh"
 #include "stages.cuh"
 
@@ -55,11 +52,9 @@ extern "C" int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv
   a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
   a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  // ACTQKV_ATTENTION=simt forces the general kernel, =tc1 the single-CTA tensor-core kernel
-  // (debugging aids; the default picks by shape).
-  const char* force = std::getenv("ACTQKV_ATTENTION");
-  const bool simt_only = force && std::strcmp(force, "simt") == 0;
-  const bool tc1_only = force && std::strcmp(force, "tc1") == 0;
+  // cfg->attention_kernel pins one kernel (for comparing kernels with each other); 0 picks by shape
+  const bool simt_only = cfg->attention_kernel == ACTQKV_ATTN_GENERAL;
+  const bool tc1_only = cfg->attention_kernel == ACTQKV_ATTN_SINGLE_CTA;
   if (!simt_only && !tc1_only && attention_tc2_supported(cfg, n_tokens)) return launch_attention_tc2(cfg, b, a, st);
   if (!simt_only && attention_tc_supported(cfg, n_tokens)) return launch_attention_tc(cfg, b, a, st);
   if (!simt_only && attention_decode_supported(cfg, n_tokens)) return launch_attention_decode(cfg, b, a, 1, nullptr, st);

@@ -81,6 +81,12 @@ __global__ void __launch_bounds__(kThreads, 3) append_kernel(AppendParams p) {
           if (g0 + u < p.n_kv_heads) d_row[size_t(g0 + u) * pt_tok * vpr] = val[u];
       }
     }
+    // The step ends inside this page: the rows after it are zeroed, so that an attention step that
+    // loads the page whole (and masks those rows) multiplies weight 0 by a finite value.
+    if (p0 + p.n_tokens < page0 + pt_tok) {
+      for (int t = t_hi + rl; t < pt_tok; t += n_rl)
+        for (int g = 0; g < p.n_kv_heads; ++g) dst[(size_t(g) * pt_tok + t) * vpr + cv] = make_uint4(0, 0, 0, 0);
+    }
     return;
   }
 

@@ -112,11 +112,17 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   const int per_split = (all_tiles + dp.n_splits - 1) / dp.n_splits;
   const int j_lo = sp * per_split;
   const int n_tiles = max(0, min(all_tiles, j_lo + per_split) - j_lo);
-  if (n_tiles == 0) {          // uniform over the CTA: more splits than tiles
+  // A split that contributes nothing says so with a log-sum-exp of minus infinity: the merge then
+  // skips its partial output, whatever an earlier call left at that place of the workspace.
+  auto mark_split_empty = [&]() {
+    if (dp.n_splits <= 1) return;
     for (int i = tid; i < nt * G; i += kThreads) {
       const int t = i / G, hh = g * G + i % G;
       dp.part_lse[((size_t(unit) * nt + t) * p.n_q_heads + hh) * dp.n_splits + sp] = -INFINITY;
     }
+  };
+  if (n_tiles == 0) {          // uniform over the CTA: more splits than tiles
+    mark_split_empty();
     return;
   }
 
@@ -142,6 +148,7 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   if (misaligned) {           // uniform: nothing was issued yet
+    mark_split_empty();
     __syncthreads();
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
     return;
@@ -417,7 +424,10 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   // ---- teardown
   tc_fence_before();
   __syncthreads();
-  if (tid == 0 && *abort_flag) set_status(p.a.status, ACTQKV_DEV_TIMEOUT);
+  if (*abort_flag) {            // a wait gave up: this split's partial result is not to be used
+    mark_split_empty();
+    if (tid == 0) set_status(p.a.status, ACTQKV_DEV_TIMEOUT);
+  }
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
@@ -486,9 +496,9 @@ int attention_decode_auto_splits(const actqkv_config* cfg, const Batch& b) {
   return std::max(1, std::min(s, 16));
 }
 
-// The caller passes pos0 of the positions BEFORE the new tokens, as for the prefill kernels; a
-// position p0 not on a 16-token boundary is served only through the local-segment rule of the
-// key layout (p0 - local_start a multiple of 16), otherwise the general kernel must be used.
+// The caller passes pos0 of the positions BEFORE the new tokens, as for the prefill kernels.  p0
+// need not sit on a page boundary: the last, partly filled page of the local segment is loaded
+// whole and the rows past p0 are masked out of the softmax (they must hold finite values).
 int launch_attention_decode(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, int n_splits,
                             void* workspace, cudaStream_t st) {
   const int U = b.units(), nt = a.n_tokens, Hq = cfg->n_q_heads, Hkv = cfg->n_kv_heads, G = Hq / Hkv;
@@ -526,13 +536,8 @@ int launch_attention_decode(const actqkv_config* cfg, const Batch& b, const Attn
   dp.part_o = static_cast<float*>(workspace);
   dp.part_lse = dp.part_o ? dp.part_o + rows * dp.n_splits * kD : nullptr;
   if (dp.n_splits > 1 && !workspace) return ACTQKV_ERR_NULL;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attention_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes)) !=
-        cudaSuccess)
-      return ACTQKV_ERR_LAUNCH;
-    attr_set = true;
-  }
+  static std::atomic<bool> opted_in[kMaxDevices];
+  if (!opt_in_shared_memory(attention_decode_kernel, int(kSmemBytes), opted_in)) return ACTQKV_ERR_LAUNCH;
   dim3 grid(dp.n_splits, Hkv, U);
   attention_decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(tm_q, tm_kw, tm_vw, tm_kp, tm_vp, p, dp);
   if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;
@@ -555,21 +560,20 @@ static __device__ __align__(256) unsigned char g_decode_scratch[ACTQKV_STATIC_SC
 
 // In host code `g_decode_scratch` is only a handle for the runtime, not a device address; the
 // address of each device's copy is asked for once, with that device current, and remembered.
-constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};
+std::atomic<void*> g_scratch_addr[actqkv::kMaxDevices];
 
 int static_scratch(void** ptr) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ACTQKV_ERR_LAUNCH;
-  if (!g_scratch_addr[dev]) {
-    void* addr = nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= actqkv::kMaxDevices) return ACTQKV_ERR_LAUNCH;
+  void* addr = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!addr) {      // two threads may both ask; they get the same answer
     if (cudaGetSymbolAddress(&addr, g_decode_scratch) != cudaSuccess || !addr) {
       (void)cudaGetLastError();
       return ACTQKV_ERR_LAUNCH;
     }
-    g_scratch_addr[dev] = addr;
+    g_scratch_addr[dev].store(addr, std::memory_order_release);
   }
-  *ptr = g_scratch_addr[dev];
+  *ptr = addr;
   return ACTQKV_OK;
 }
 
@@ -605,9 +609,10 @@ extern "C" int actqkv_decode_attention_static(const actqkv_config* cfg, const ac
   a.q = q; a.k_win = k_win; a.v_win = v_win; a.k_pages = k_pages; a.v_pages = v_pages;
   a.page_table = page_table; a.pos0 = pos0; a.sel_idx = sel_idx; a.sel_count = sel_count;
   a.out = out; a.lse = lse; a.status = status; a.n_tokens = n_tokens;
-  // Nothing in the scratch has to start at zero: every split writes its log-sum-exp (minus
-  // infinity when it holds no tile) and the merge reads a partial output only where that value
-  // is finite, so what an earlier call left behind is never read.
+  // Nothing in the scratch has to start at zero: every split writes its log-sum-exp -- minus
+  // infinity when it holds no tile, or when it gave up on a bounded wait -- and the merge reads a
+  // partial output only where that value is finite, so what an earlier call left behind is never
+  // read.
   return launch_attention_decode(cfg, b, a, n_splits, scratch, reinterpret_cast<cudaStream_t>(stream));
 }
 

@@ -196,13 +196,13 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   ks.g_init = geo.init_len / 16;
   ks.g_sel = c * ks.gpb;
   const int64_t local_len = geo.p0 - geo.local_start;
-  ks.g_past = ks.g_init + ks.g_sel + int(local_len / 16);
+  ks.g_past = ks.g_init + ks.g_sel + int((local_len + 15) / 16);   // the last local page may be partly filled
   ks.n_cand = geo.n_cand; ks.n_init = p.n_init; ks.block = p.block; ks.max_pages = p.max_pages;
   ks.n_phys_pages = p.n_phys_pages; ks.page_base = layer_local * p.n_phys_pages;
   ks.page_oob = p.n_layers * p.n_phys_pages;             // beyond the tensor: zero fill
   ks.local_start = geo.local_start;
-  const bool misaligned = (local_len % 16) != 0 || smem_short;
-  const int n_past = ks.g_past * 16;
+  const bool misaligned = smem_short;
+  const int n_past = geo.init_len + c * p.block + int(local_len);     // exact: the tail of the last page is masked
   const int past_tiles = (n_past + kBN - 1) / kBN;
   const int n_tiles = past_tiles + mt + 1;
 
@@ -605,13 +605,8 @@ int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArg
   p.n_phys_pages = cfg->n_phys_pages; p.n_layers = b.n_layers; p.out_bf16 = cfg->out_dtype == ACTQKV_BF16;
   const float scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.f / sqrtf(float(kD));
   p.scale_log2 = scale * 1.4426950408889634f;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes)) !=
-        cudaSuccess)
-      return ACTQKV_ERR_LAUNCH;
-    attr_set = true;
-  }
+  static std::atomic<bool> opted_in[kMaxDevices];
+  if (!opt_in_shared_memory(attention_tc2_kernel, int(kSmemBytes), opted_in)) return ACTQKV_ERR_LAUNCH;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(Hq, nt / kBM, U);
   lc.blockDim = dim3(kThreads, 1, 1);

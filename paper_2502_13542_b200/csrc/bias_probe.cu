@@ -41,6 +41,7 @@ struct BiasProbeParams {
   int stats_mode;
   int do_bias;    // compute statistics + phi (else phi_l1 is an input)
   int do_probe;   // compute probes
+  int mean_pool;  // uniform token weights (the mean-pooling probe) instead of Eq. 9's
   int32_t* status;
 };
 
@@ -324,7 +325,7 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
 #pragma unroll
       for (int rk = 0; rk < kMaxCluster; ++rk)
         if (rk >= y * S && rk < (y + 1) * S) { t += tot[rk]; u2 += uu[rk]; q2 += qq[rk]; }
-      return t > 0.f ? u2 / t : q2 / float(W);      // all-zero bias: uniform weights
+      return (t > 0.f && !p.mean_pool) ? u2 / t : q2 / float(W);      // all-zero bias: uniform weights
     };
     p.probe_qh[hd + tid] = head_probe(cy > 1 ? hy : 0);
     if (hy == 0) {
@@ -679,7 +680,7 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
         float t = 0.f;
         for (int i = 0; i < kStreamThreads / 32; ++i) t += red_s[i];
         const float qsum = p.do_bias ? qsum_s[tid] : sum_b[tid];
-        p.probe_qh[hd + tid] = t > 0.f ? sum_a[tid] / t : qsum / float(W);   // all-zero bias: uniform weights
+        p.probe_qh[hd + tid] = (t > 0.f && !p.mean_pool) ? sum_a[tid] / t : qsum / float(W);   // all-zero bias: uniform weights
       }
     }
     __syncthreads();
@@ -694,6 +695,24 @@ __global__ void probe_kv_kernel(const float* probe_qh, float* probe_kv, int n_q_
     for (int y = 0; y < group; ++y) acc += probe_qh[(size_t(unit) * n_q_heads + g * group + y) * D + ch];
     probe_kv[(size_t(unit) * n_kv_heads + g) * D + ch] = acc / float(group);
   }
+}
+
+// A step of one token: the probe of a query head is the token's query itself, whatever the weights
+// (Eq. 9 with a single term); the KV-head probe is the mean over the group.  One block per
+// (unit, KV head), one thread per channel.
+template <typename T>
+__global__ void probe_one_token_kernel(const T* __restrict__ q, float* __restrict__ probe_qh, float* __restrict__ probe_kv,
+                                       int n_q_heads, int n_kv_heads, int group) {
+  grid_dependency_wait();
+  const int unit = blockIdx.x / n_kv_heads, g = blockIdx.x - unit * n_kv_heads, D = blockDim.x, ch = threadIdx.x;
+  float acc = 0.f;
+  for (int y = 0; y < group; ++y) {
+    const size_t i = (size_t(unit) * n_q_heads + g * group + y) * D + ch;
+    const float x = to_f32(q[i]);
+    probe_qh[i] = x;
+    acc += x;
+  }
+  probe_kv[(size_t(unit) * n_kv_heads + g) * D + ch] = acc / float(group);
 }
 
 // Returns 1 when the shape does not suit the streaming kernel (the caller takes the cluster kernel).
@@ -803,7 +822,19 @@ int run(const actqkv_config* cfg, const actqkv_batch* batch, BiasProbeParams& p,
   p.group = cfg->n_q_heads / cfg->n_kv_heads;
   p.var_eps = cfg->var_eps > 0.f ? cfg->var_eps : 1e-12f;
   p.stats_mode = cfg->stats_mode;
+  p.mean_pool = cfg->probe_mode == ACTQKV_PROBE_MEAN_POOL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (p.n_tokens == 1 && p.do_probe && !p.do_bias) {
+    // one token: every weighting gives probe_qh = q (the decode-stage probe, Sec. 4.2)
+    const int n = b.units() * cfg->n_kv_heads;
+    if (cfg->dtype == ACTQKV_BF16)
+      probe_one_token_kernel<__nv_bfloat16><<<n, cfg->head_dim, 0, st>>>(static_cast<const __nv_bfloat16*>(p.q), p.probe_qh,
+                                                                         p.probe_kv, cfg->n_q_heads, cfg->n_kv_heads, p.group);
+    else
+      probe_one_token_kernel<float><<<n, cfg->head_dim, 0, st>>>(static_cast<const float*>(p.q), p.probe_qh, p.probe_kv,
+                                                                 cfg->n_q_heads, cfg->n_kv_heads, p.group);
+    return launch_status();
+  }
   return cfg->dtype == ACTQKV_BF16 ? launch<__nv_bfloat16>(cfg, b, p, st) : launch<float>(cfg, b, p, st);
 }
 
@@ -835,7 +866,8 @@ extern "C" int actqkv_probe_query(const actqkv_config* cfg, const actqkv_batch* 
                                   int32_t* status, void* stream) {
   if (!cfg) return ACTQKV_ERR_NULL;
   ACTQKV_REQUIRE_PTR(q);
-  ACTQKV_REQUIRE_PTR(phi_l1);
+  if (n_tokens == 1) ACTQKV_OPTIONAL_PTR(phi_l1);    // a single token's weight is 1 whatever phi says
+  else ACTQKV_REQUIRE_PTR(phi_l1);
   ACTQKV_REQUIRE_PTR(probe_qh);
   ACTQKV_REQUIRE_PTR(probe_kv);
   BiasProbeParams p = {};

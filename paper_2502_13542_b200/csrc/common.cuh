@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "actqkv.h"
 
 namespace actqkv {
@@ -26,6 +28,8 @@ inline int check_config(const actqkv_config* c, const Batch& b) {
   if (!c) return ACTQKV_ERR_NULL;
   if (c->dtype != ACTQKV_F32 && c->dtype != ACTQKV_BF16) return ACTQKV_ERR_DTYPE;
   if (c->out_dtype != ACTQKV_F32 && c->out_dtype != ACTQKV_BF16) return ACTQKV_ERR_DTYPE;
+  if (c->probe_mode != ACTQKV_PROBE_ACTIVATION && c->probe_mode != ACTQKV_PROBE_MEAN_POOL) return ACTQKV_ERR_SHAPE;
+  if (c->attention_kernel < ACTQKV_ATTN_AUTO || c->attention_kernel > ACTQKV_ATTN_SINGLE_CTA) return ACTQKV_ERR_SHAPE;
   if (c->head_dim != 64 && c->head_dim != 128) return ACTQKV_ERR_SHAPE;
   if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_q_heads % c->n_kv_heads) return ACTQKV_ERR_SHAPE;
   if (c->n_q_heads / c->n_kv_heads > 8) return ACTQKV_ERR_SHAPE;
@@ -65,6 +69,25 @@ inline void prefer_max_shared(Kernel kern) {
 inline void allow_early_launch(cudaLaunchAttribute& a) {
   a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   a.val.programmaticStreamSerializationAllowed = 1;
+}
+
+// A kernel that needs more than 48 KiB of dynamic shared memory must opt in, and the opt-in
+// belongs to the device that was current when it was made.  `done` is a per-kernel table with one
+// flag per device ordinal; two host threads that race on a device's first launch both make the
+// (idempotent) call.
+constexpr int kMaxDevices = 64;
+template <typename Kernel>
+inline bool opt_in_shared_memory(Kernel kern, int bytes, std::atomic<bool> (&done)[kMaxDevices]) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return false;
+  const bool tracked = dev < kMaxDevices;
+  if (tracked && done[dev].load(std::memory_order_acquire)) return true;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  if (tracked) done[dev].store(true, std::memory_order_release);
+  return true;
 }
 
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? ACTQKV_OK : ACTQKV_ERR_LAUNCH; }

@@ -279,13 +279,20 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
-// 8 bf16 values (16 bytes) to 8 fp16 values, exact for magnitudes in [2^-14, 65504].
+// Saturating form: finite values beyond the fp16 range become +-65504 instead of infinity.
+__device__ __forceinline__ uint32_t pack_f16_sat(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// 8 bf16 values (16 bytes) to 8 fp16 values, exact for magnitudes in [2^-14, 65504]; larger finite
+// magnitudes saturate at 65504 (an infinity would turn weight-0 products into NaN).
 __device__ __forceinline__ uint4 bf16x8_to_f16x8(uint4 v) {
   uint4 r;
-  r.x = pack_f16(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
-  r.y = pack_f16(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
-  r.z = pack_f16(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u));
-  r.w = pack_f16(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
+  r.x = pack_f16_sat(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u));
+  r.y = pack_f16_sat(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+  r.z = pack_f16_sat(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u));
+  r.w = pack_f16_sat(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
   return r;
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
@@ -393,16 +400,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 inline EncodeTiledFn get_encode() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  // initialised once, by whichever host thread gets here first (C++11 guarantees the others wait)
+  static const EncodeTiledFn fn = [] {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
-  }
+      return reinterpret_cast<EncodeTiledFn>(sym);
+    return EncodeTiledFn(nullptr);
+  }();
   return fn;
 }
 

@@ -266,3 +266,20 @@ def to_pages(spec: WorkloadSpec, x_tokens: np.ndarray, page_table: np.ndarray,
     pages = np.zeros((n_phys_pages, hkv, pt, d), x_tokens.dtype)
     pages[page_table[:n_log]] = x_tokens.reshape(n_log, pt, hkv, d).transpose(0, 2, 1, 3)
     return pages
+
+
+# ----------------------------------------------------------------------------
+# host <-> device plumbing (no arithmetic: exact conversions only)
+# ----------------------------------------------------------------------------
+def to_device(x, spec: WorkloadSpec, device="cuda"):
+    """A generated float32 array as a device tensor of the workload's dtype (exact: bf16
+    workloads are generated on the bf16 grid)."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(device)
+    return t.to(torch.bfloat16) if spec.dtype == "bf16" else t
+
+
+def to_numpy(t) -> np.ndarray:
+    """A device tensor as a host array (float32, or float64 for float64 tensors)."""
+    import torch
+    return t.detach().to(torch.float32).cpu().numpy() if t.dtype != torch.float64 else t.detach().cpu().numpy()

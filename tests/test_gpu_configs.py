@@ -76,14 +76,109 @@ def test_tiny_stack32_paper_temperature(B):
     print("tiny stack, beta = 1: per-layer counts at the last window", counts[-1][1])
 
 
-def test_llama_stack32_sharpened_density(B):
-    """32 layers of the LLaMA3-8B shape (bf16, paged) at 16k context with a sharpened softmax
-    (beta = 32) so that the per-layer counts really differ and the cap binds; tensor-core
-    attention of the last window checked on layers 0, 13 and 31."""
-    spec = wl.llama3_8b_stack32().replace(context=16384)
-    counts = _stack(B, spec, 32.0, attention_layers={0, 13, 31}, check_windows=set(range(0, 32, 3)) | {31})
-    late = counts[-1][1]
-    assert len(set(late)) > 2, late
+def test_llama_stack32_32k_paper_and_sharpened_temperature(B):
+    """The 32-layer stack at its stated size: LLaMA3-8B shape, context 32768 (64 windows), k = 32,
+    cap 64, all layers batched per call, at beta = 1 (the paper's softmax) AND beta = 32 (counts
+    vary by layer and hit the cap).  Both temperatures share the bias / probe / score stages (they
+    do not depend on beta); the beta = 32 cut-off runs on a second set of selection buffers.
+    Scores and densities at every checked window (every 4th, the first two and the last), counts
+    at every window, block sets at the checked ones, tensor-core attention of the last window on
+    layers {0, 13, 31} for both temperatures."""
+    import torch
+    spec = wl.llama3_8b_stack32()
+    L, Hkv = spec.n_layers, spec.n_kv_heads
+    att_layers = {0, 13, 31}
+    cfg1 = B.make_config(spec, beta=1.0, out_dtype=B.F32)
+    cfg32 = B.make_config(spec, beta=32.0, out_dtype=B.F32)
+    pt = wl.shuffled_page_table(spec, spec.context)
+    st = B.RetrievalState(cfg1, n_seq=1, n_layers=L, page_table=pt[None, :])
+    budget32 = torch.zeros_like(st.budget_state)
+    scores32, theta32 = torch.zeros_like(st.scores), torch.zeros_like(st.theta)
+    sel_idx32, sel_count32, real32 = torch.full_like(st.sel_idx, -1), torch.zeros_like(st.sel_count), torch.zeros_like(st.budget_real)
+    chain1 = orc.BudgetChain(L, spec.k_blocks, spec.cap_blocks, "streaming")
+    chain32 = orc.BudgetChain(L, spec.k_blocks, spec.cap_blocks, "streaming")
+    runners = [pu.OracleRunner(spec, layer=l, chain=chain1, beta=1.0) for l in range(L)]
+    out = torch.zeros(L, spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
+    out32 = torch.zeros_like(out)
+    T = spec.n_windows
+    tally = dict(windows=0, sets=0, near=0, fragile=0, att=0, worst_att=0.0)
+    last_counts = None
+    for t in range(T):
+        last = t == T - 1
+        check = last or t < 2 or t % 4 == 3
+        qs, ks, vs, res, res32 = [], [], [], [], []
+        for l in range(L):
+            q = wl.gen_q(spec, l, t)
+            k, v = wl.gen_kv(spec, l, t)
+            qs.append(q); ks.append(k); vs.append(v)
+            r = runners[l].step(q, k, v, attention=last and l in att_layers)
+            res.append(r)
+            th = orc.information_density(r["scores"], 32.0)
+            c, b_real, fragile = chain32.grant(l, th, r["n"])
+            r32 = dict(c=c, b_real=b_real, fragile=fragile, theta=th)
+            if check:
+                picks = [orc.select_blocks(r["scores"][g], c) for g in range(Hkv)]
+                r32.update(sel=[x[0] for x in picks], tau=[x[1] for x in picks], near=[x[2] for x in picks])
+                if last and l in att_layers:
+                    state = runners[l].state
+                    r32["out"], _ = orc.retrieval_attention(q, k, v, state.k_cache, state.v_cache, r["p0"], r32["sel"],
+                                                            spec.n_init, spec.block, spec.n_local_prev)
+            res32.append(r32)
+        dq, dk, dv = (pu.to_device(np.stack(x), spec) for x in (qs, ks, vs))
+        st.step(dq, dk, dv, out, advance=False)
+        B.score_select(cfg32, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, budget32, scores32,
+                       theta32, sel_idx32, sel_count32, real32, st.status)
+        if last:
+            B.retrieval_attention(cfg32, st.batch, dq, dk, dv, spec.window, st.k_pages, st.v_pages, st.page_table,
+                                  st.pos0, sel_idx32, sel_count32, out32, None, st.status)
+        st.set_positions([(t + 1) * spec.window])
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        n = res[0]["n"]
+        for beta, rr, cnt, idx, th_gpu, o_gpu in ((1.0, res, st.sel_count, st.sel_idx, st.theta, out),
+                                                  (32.0, res32, sel_count32, sel_idx32, theta32, out32)):
+            tag = f"{spec.name} beta={beta} window {t}"
+            got_c = cnt.cpu().numpy().tolist()
+            want_c = [r["c"] for r in rr]
+            if any(r["fragile"] for r in rr):
+                tally["fragile"] += 1
+                # a rounding decision on the boundary: the later layers of this step inherit the
+                # difference, so follow the device from here on
+                assert sum(abs(a - b) for a, b in zip(got_c, want_c)) <= 2 * sum(r["fragile"] for r in rr), tag
+                chain = chain1 if beta == 1.0 else chain32
+                chain.b_rem = float(budget32[0, 0] if beta == 32.0 else st.budget_state[0, 0])
+                continue
+            assert got_c == want_c, tag
+            if not (check and n):
+                continue
+            th = pu.to_numpy(th_gpu)
+            for l in range(L):
+                if beta == 1.0:
+                    pu.assert_rel(pu.to_numpy(st.scores[l, :, :n]), res[l]["scores"], 1.0, f"{tag} layer {l} scores")
+                pu.assert_rel(th[l], rr[l]["theta"], 1e-30, f"{tag} layer {l} theta", tol=2e-4 if beta > 1 else pu.REL_TOL)
+                r_full = dict(res[l], **rr[l]) if beta != 1.0 else rr[l]
+                nd = pu.compare_selection(pu.to_numpy(idx[l]).astype(np.int64), got_c[l], r_full, f"{tag} layer {l}")
+                assert nd >= 0
+                tally["sets"] += 1
+                tally["near"] += nd
+                if last and l in att_layers and nd == 0:
+                    mx, _ = pu.assert_attention(pu.to_numpy(o_gpu[l]), rr[l]["out"], f"{tag} layer {l} attention")
+                    tally["att"] += 1
+                    tally["worst_att"] = max(tally["worst_att"], mx)
+            if last:
+                last_counts = (last_counts or {})
+                last_counts[beta] = want_c
+        tally["windows"] += 1
+    print("stack32 at 32k:", tally)
+    last_counts = last_counts or {}
+    print("  counts at the last window, beta = 1 :", last_counts.get(1.0))
+    print("  counts at the last window, beta = 32:", last_counts.get(32.0))
+    print("  exp(theta) per layer at the last window (beta = 1):",
+          [round(float(np.exp(np.mean(r["theta"]))), 2) for r in res])
+    assert tally["att"] >= 5                                   # of 6 (3 layers x 2 temperatures)
+    assert abs(float(st.budget_state[0, 0]) - chain1.b_rem) < 1e-9
+    c32 = last_counts.get(32.0) or sel_count32.cpu().numpy().tolist()
+    assert len(set(c32)) > 2 and max(c32) == spec.cap_blocks   # counts vary by layer, the cap binds
 
 
 def test_long_131k_sweep(B):
@@ -97,7 +192,7 @@ def test_long_131k_sweep(B):
     run = pu.OracleRunner(spec)
     out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.float32, device="cuda")
     att = {0, 1, 31, 32, 33, 127, 255}
-    near = 0
+    near = att_checked = 0
     for t in range(spec.n_windows):
         q = wl.gen_q(spec, 0, t)
         k, v = wl.gen_kv(spec, 0, t)
@@ -117,6 +212,8 @@ def test_long_131k_sweep(B):
         near += nd
         if t in att and nd == 0:
             pu.assert_attention(pu.to_numpy(out), res["out"], tag + " attention")
+            att_checked += 1
+    assert att_checked >= len(att) - 1, f"attention compared at only {att_checked} of {len(att)} sampled windows"
     sel = pu.to_numpy(st.sel_idx[0]).astype(int)
     for g in range(spec.n_kv_heads):
         assert set(wl.planted_blocks(spec, 0)[g]) <= set(sel[g])
@@ -217,7 +314,7 @@ def test_decode_batch_fixed_probes(B):
 
 
 @pytest.mark.parametrize("n_new", [1, 5, 32])
-def test_decode_attention_splits_match_general_kernel(B, monkeypatch, n_new):
+def test_decode_attention_splits_match_general_kernel(B, n_new):
     """The tensor-core decode kernel, unsplit and with the key stream cut into 2, 5, 16 and the
     automatic number of shares (workspace + merge kernel), against the general fp32 kernel on the
     same state: ragged position (the last cache page partly filled), 512 local tokens, steps of
@@ -243,11 +340,10 @@ def test_decode_attention_splits_match_general_kernel(B, monkeypatch, n_new):
                    st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
     shape = (1, n_new, spec.n_q_heads, spec.head_dim)
     ref, ref_lse = torch.zeros(shape, device="cuda"), torch.zeros(spec.n_q_heads, n_new, device="cuda")
-    monkeypatch.setenv("ACTQKV_ATTENTION", "simt")
-    B.retrieval_attention(cfg, st.batch, q, k, v, n_new, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+    cfg_gen = B.make_config(spec, out_dtype=B.F32, max_context=8192, attention_kernel=B.ATTN_GENERAL)
+    B.retrieval_attention(cfg_gen, st.batch, q, k, v, n_new, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
                           st.sel_count, ref, ref_lse, st.status)
     torch.cuda.synchronize()
-    monkeypatch.delenv("ACTQKV_ATTENTION")
     auto = B.decode_splits(cfg, st.batch)
     assert auto >= 8                                      # 8 (unit, KV head) pairs on a GPU of ~148 SMs
     for splits in (1, 2, 5, 16, 0):

@@ -440,3 +440,42 @@ def test_planted_block_recall_tiny_config():
                                    sp.n_init, sp.block)
     want = orc.full_causal_attention(q, st.k_cache, st.v_cache, p0)
     assert np.allclose(o, want, rtol=1e-10, atol=1e-12)
+
+
+def test_window_retrieval_variant_switches_reduce_to_library_routines():
+    """The switches of the whole-path function: window-only statistics are numpy's mean and
+    unbiased variance of the CURRENT window alone (no history), and the mean-pooling probe
+    (Sec. 1 of the paper: the probe its baselines use) is numpy's mean over the window's tokens
+    followed by the mean over each KV head's group of query heads."""
+    sp = wl.tiny_pr1()
+    for stats_mode, probe_mode in (("window_only", "activation"), ("cumulative", "mean_pool")):
+        st = orc.LayerState(sp.n_q_heads, sp.n_kv_heads, sp.head_dim)
+        ch = orc.BudgetChain(1, sp.k_blocks, sp.cap_blocks)
+        for t in range(3):
+            q = wl.gen_q(sp, 0, t)
+            k, v = wl.gen_kv(sp, 0, t)
+            res = orc.window_retrieval(st, ch, 0, q, k, v, n_init=sp.n_init, block=sp.block, n_repr=sp.n_repr,
+                                       dtype=sp.dtype, attention=False, stats_mode=stats_mode,
+                                       probe_mode=probe_mode)
+        q64 = q.astype(np.float64)
+        if stats_mode == "window_only":
+            assert np.allclose(res["zbar"], q64.mean(axis=0), rtol=1e-12, atol=1e-14)
+            assert np.allclose(res["sigma2"], q64.var(axis=0, ddof=1), rtol=1e-12)
+            assert st.stats.count == 0                      # the running statistics are left alone
+        else:
+            hist = np.concatenate([wl.gen_q(sp, 0, i) for i in range(3)]).astype(np.float64)
+            assert np.allclose(res["sigma2"], hist.var(axis=0, ddof=1), rtol=1e-12)
+        if probe_mode == "mean_pool":
+            want_qh = q64.mean(axis=0)
+            assert np.allclose(res["probe_qh"], want_qh, rtol=1e-12, atol=1e-14)
+            want_kv = want_qh.reshape(sp.n_kv_heads, sp.group, sp.head_dim).mean(axis=1)
+            assert np.allclose(res["probe_kv"], want_kv, rtol=1e-12, atol=1e-14)
+        else:
+            assert not np.allclose(res["probe_qh"], q64.mean(axis=0), rtol=1e-3)   # Eq. 9 is not a plain mean here
+
+
+def test_one_token_probe_is_the_query_itself():
+    """Decode (Sec. 4.2): with a single token Eq. 9 has one term of weight 1, whatever phi is."""
+    q = rng(3).standard_normal((1, 4, 8))
+    for a in (np.ones((1, 4)), np.full((1, 4), 7.5), np.zeros((1, 4))):
+        assert np.allclose(orc.probe_query(q, a), q[0], rtol=0, atol=0)
