@@ -128,6 +128,11 @@ def stage_bytes(spec, p0):
     }
 
 
+def stage_free_step_us(stage_all) -> float:
+    """Sum of the median stage times of one step (an upper bound of the overlapped step)."""
+    return float(sum(np.median(v) for v in stage_all.values()))
+
+
 def max_over_ranks(x: float, device=None) -> float:
     """The slowest rank's value (all ranks get it); the identity when there is one process."""
     import torch
@@ -146,9 +151,20 @@ def job_throughput(units_per_rank_step: int, world: int, ms_per_step: float) -> 
 
 
 # ------------------------------------------------------------------------------------------
-def build_states(spec, n_copies, device):
+def l2_flusher(device, mbytes=512):
+    """Returns a function that reads a buffer several times the L2 size: afterwards nothing a
+    kernel reads is in L2, and the lines it leaves behind are clean (no write-back traffic lands in
+    the next timed launch)."""
+    import torch
+    scratch = torch.zeros(mbytes << 20, dtype=torch.uint8, device=device)
+    return lambda: scratch.view(torch.int32).sum()
+
+
+def build_states(spec, n_copies, device, sweep_times=None, flush=None):
     """Prefills one layer up to the last window on the GPU, then clones the state into
-    n_copies physically distinct copies.  Returns (cfg, states, inputs of the last window)."""
+    n_copies physically distinct copies.  Returns (cfg, states, inputs of the last window).
+    With sweep_times (a list) every window's step is timed with CUDA events after an L2 flush and
+    its microseconds are appended: the prefill sweep itself is the measurement."""
     import torch
     from paper_2502_13542_b200 import binding as B
     from paper_2502_13542_b200 import workloads as wl
@@ -157,12 +173,21 @@ def build_states(spec, n_copies, device):
     base = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :], device=device)
     out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=device)
     T = spec.n_windows
+    evs = []
     for t in range(T - 1):
         q = wl.to_device(wl.gen_q(spec, 0, t)[None], spec, device)
         k, v = wl.gen_kv(spec, 0, t)
         k, v = wl.to_device(k[None], spec, device), wl.to_device(v[None], spec, device)
-        base.step(q, k, v, out)
+        if sweep_times is not None:
+            flush()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(); base.step(q, k, v, out, overlap_append=True); e1.record()
+            evs.append((e0, e1))
+        else:
+            base.step(q, k, v, out)
     torch.cuda.synchronize()
+    if sweep_times is not None:
+        sweep_times.extend(1e3 * a.elapsed_time(b) for a, b in evs)
     q = wl.to_device(wl.gen_q(spec, 0, T - 1)[None], spec, device)
     k, v = wl.gen_kv(spec, 0, T - 1)
     k, v = wl.to_device(k[None], spec, device), wl.to_device(v[None], spec, device)
@@ -196,8 +221,21 @@ def run_ours(args):
     spec = wl.llama3_8b_layer()
     p0 = (spec.n_windows - 1) * spec.window
     n_copies = args.copies
-    cfg, states, inputs = build_states(spec, n_copies, device)
+    extras = world == 1 and not args.headline_only
+    sweep_us = [] if extras else None
+    cfg, states, inputs = build_states(spec, n_copies, device, sweep_times=sweep_us,
+                                       flush=l2_flusher(device) if extras else None)
     peaks = load_peaks()
+    # One untimed step on the first copy, kept for the comparison with the oracle (the copies stand
+    # exactly where the prefill sweep left the layer, so this is the sweep's last window).
+    parity_sample = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        st0 = states[0]
+        q0, k0, v0, out0 = inputs[0]
+        st0.step(q0, k0, v0, out0, advance=False)
+        torch.cuda.synchronize()
+        parity_sample = {"out": out0.float().cpu().numpy(), "sel": st0.sel_idx[0].cpu().numpy().astype(np.int64),
+                         "c": int(st0.sel_count.item())}
 
     side = torch.cuda.Stream(device=device)
 
@@ -253,27 +291,36 @@ def run_ours(args):
     sampler.start()
     if args.profile_region:
         torch.cuda.profiler.start()          # cudaProfilerStart: lets a profiler capture the timed region only
-    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        one_step(args.warmup + i)
-    e1.record()
+    # The timed region of K steps is repeated `reps` times (each bracketed by a barrier and a device
+    # synchronisation): a K-step region lasts a millisecond or two, so one sample would say little.
+    # ms_per_step is the median repetition; min and max are reported beside it.
+    rep_ms, step_idx = [], args.warmup
+    for _ in range(max(1, args.reps)):
+        barrier()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            one_step(step_idx + i)
+        e1.record()
+        step_idx += args.steps
+        barrier()
+        rep_ms.append(max_over_ranks(e0.elapsed_time(e1), device) / args.steps)
     if args.profile_region:
-        torch.cuda.synchronize()
         torch.cuda.profiler.stop()
     sampler.sample()
-    barrier()
     clocks = sampler.stop()
-    ms_total = max_over_ranks(e0.elapsed_time(e1), device)
-    ms_step = ms_total / args.steps
+    ms_step = float(np.median(rep_ms))
     value = job_throughput(spec.window, world, ms_step)
+    step_stats = {"reps": len(rep_ms), "steps_per_rep": args.steps, "median_ms": ms_step,
+                  "min_ms": float(np.min(rep_ms)), "max_ms": float(np.max(rep_ms))}
 
     # instrumented pass: per-stage device time with events around each call
     events = {}
-    for i in range(args.steps):
+    for i in range(max(args.steps, 20)):
         one_step(args.warmup + i, events)
     torch.cuda.synchronize()
-    stage_us = {k: 1e3 * float(np.mean([a.elapsed_time(b) for a, b in v])) for k, v in events.items()}
+    stage_all = {k: [1e3 * a.elapsed_time(b) for a, b in v] for k, v in events.items()}
+    stage_us = {k: float(np.mean(v)) for k, v in stage_all.items()}
     assert all(int(st.status.item()) == 0 for st in states), "device status set during the bench"
 
     c_sel = int(states[0].sel_count.item())
@@ -284,7 +331,8 @@ def run_ours(args):
                 "unit": "TFLOP/s", "frac": att_tflops / peak, "traffic": attention_traffic(),
                 "peak_source": peaks["source"] + " burst bf16 (cuBLAS)", "flops_per_launch": flops}
     sb = stage_bytes(spec, p0)
-    stages = {k: {"us": v} for k, v in stage_us.items()}
+    stages = {k: {"us": v, "median_us": float(np.median(stage_all[k])), "min_us": float(np.min(stage_all[k]))}
+              for k, v in stage_us.items()}
     stages["bias_probe"]["GBps"] = sb["bias_probe"] / stage_us["bias_probe"] / 1e3
     stages["score_select"]["GBps"] = (sb["score"] + sb["select"]) / stage_us["score_select"] / 1e3
     stages["append"]["GBps"] = sb["append"] / stage_us["append"] / 1e3
@@ -352,6 +400,77 @@ def run_ours(args):
            "mode": "copies of neighbouring steps overlap the step's kernels (three streams, one host wait at the end)",
            "one_step_at_a_time": world * spec.window * e2e_steps / t_sync}
 
+    secondary = {}
+    if extras:
+        # ---- sustained: the same step loop for about two seconds with the clock sampler running, and
+        # the attention alone for about one second (its fraction is then taken against the sustained peak)
+        def sustained(fn, seconds, est_ms):
+            n = max(50, int(seconds / (est_ms * 1e-3)))
+            smp = ClockSampler(local, period=0.02)
+            torch.cuda.synchronize()
+            smp.start()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(n):
+                fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            ck = smp.stop()
+            ms = a.elapsed_time(b) / n
+            return ms, n, ck
+
+        ms_s, n_s, ck_s = sustained(lambda i: one_step(i), 2.0, ms_step)
+
+        def att_only(i):
+            st = states[i % n_copies]
+            q_, k_, v_, o_ = inputs[i % n_copies]
+            B.retrieval_attention(cfg, st.batch, q_, k_, v_, spec.window, st.k_pages, st.v_pages, st.page_table,
+                                  st.pos0, st.sel_idx, st.sel_count, o_, None, st.status)
+        ms_a, n_a, ck_a = sustained(att_only, 1.0, stage_us["attention"] * 1e-3)
+        tf_a = flops / (ms_a * 1e-3) / 1e12
+        secondary["sustained"] = {
+            "step": {"seconds": ms_s * n_s * 1e-3, "steps": n_s, "ms_per_step": ms_s, "tokens_per_s_layer": spec.window / (ms_s * 1e-3),
+                     "sm_mhz_median": ck_s["sm_mhz"], "ms_x_mhz": ms_s * (ck_s["sm_mhz"] or 0), "reasons": ck_s["reasons"]},
+            "attention": {"seconds": ms_a * n_a * 1e-3, "launches": n_a, "us_per_launch": ms_a * 1e3, "TFLOPs": tf_a,
+                          "frac_of_sustained_bf16_peak": tf_a / peaks["bf16_tflops_sustained"],
+                          "sm_mhz_median": ck_a["sm_mhz"], "reasons": ck_a["reasons"]}}
+        # ---- the whole 32k prefill sweep, window by window (timed while the states were built)
+        sweep_all = list(sweep_us) + [stage_free_step_us(stage_all)]
+        secondary["sweep_32k"] = {"windows": len(sweep_all), "sum_ms": float(np.sum(sweep_all)) * 1e-3,
+                                  "tokens_per_s_layer": spec.context / (float(np.sum(sweep_all)) * 1e-6),
+                                  "first_window_us": sweep_all[0], "last_window_us": sweep_all[-1],
+                                  "note": "every window timed alone with CUDA events after an L2 flush; the last one is the headline step"}
+        sweep_all[-1] = ms_step * 1e3
+        secondary["sweep_32k"]["sum_ms"] = float(np.sum(sweep_all)) * 1e-3
+        secondary["sweep_32k"]["tokens_per_s_layer"] = spec.context / (float(np.sum(sweep_all)) * 1e-6)
+        secondary["sweep_32k"]["last_window_us"] = sweep_all[-1]
+        # ---- batched shapes of the memory-bound stages, the full-size score launch, the 131k sweep
+        del states, inputs
+        torch.cuda.empty_cache()
+        iters = 20
+        s32 = measure_stack32(iters, device)
+        torch.cuda.empty_cache()
+        d16 = measure_decode16(iters, device)
+        torch.cuda.empty_cache()
+        sfull = measure_score_full(iters, device)
+        torch.cuda.empty_cache()
+
+        def pick(d, name, alias=None):
+            x = d["stages"][name]
+            return {"us": x["us"], "min_us": x["min_us"], "bytes": x["bytes"], "GBps": x["GBps"],
+                    "frac_of_measured_hbm": x["frac_of_measured_hbm"]}
+        secondary["stages_batched"] = {
+            "stack32": {"workload": s32["workload"], "bias_probe": pick(s32, "bias_probe"),
+                        "score_select": pick(s32, "score_select"), "score_blocks": pick(s32, "score_blocks"),
+                        "select_cutoff": pick(s32, "select_cutoff"), "append": pick(s32, "append")},
+            "decode16": {"workload": d16["workload"], "score_select": pick(d16, "score_select"),
+                         "score_blocks": pick(d16, "score_blocks"), "select_cutoff": pick(d16, "select_cutoff"),
+                         "attention_decode": pick(d16, "attention_decode"), "keys_per_head": d16["keys_per_head"]},
+            "score_full_decode_step": sfull, "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "cold_l2": "512 MB read through L2 before every timed launch; median of 20 launches"}
+        secondary["long131k"] = measure_long131k(device, peaks)
+        torch.cuda.empty_cache()
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -360,11 +479,12 @@ def run_ours(args):
                                "Hq=32 Hkv=8 D=128 W=512 B=128 r=4 n_init=128 k=cap=32, bf16 16-token pages",
                    "cold_l2": f"{n_copies} distinct layer-state copies rotated (inputs larger than L2)",
                    "selected_blocks": c_sel, "parallelism": f"independent layers x{world}", "streams": "append on a second stream, joined every step"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "roofline": roofline, "stages": stages,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps * len(rep_ms),
+        "roofline": roofline, "stages": stages, "step_stats": step_stats,
     }
+    line.update(secondary)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(spec, budget_s=args.cpu_budget)
+        line["cpu_baseline"], line["parity"] = cpu_baseline(spec, budget_s=args.cpu_budget, gpu=parity_sample)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -413,11 +533,39 @@ def _oracle_state(spec):
     return (run.state, run.chain, run.table), q, k, v
 
 
-def cpu_baseline(spec, budget_s=12.0):
+def oracle_parity(spec, st_cache, q, k, v, gpu, head=3):
+    """The timed configuration against the oracle: the selected block sets of every KV head, and the
+    bf16-stored attention output of the query heads of one KV head, element by element."""
+    from oracle import actqkv_oracle as orc
+    state, chain, table = st_cache
+    s2 = state.stats.copy()
+    s2.update(q)
+    _, a = orc.activation_bias(q, s2.mean, s2.variance())
+    pkv = orc.kv_head_probe(orc.probe_query(q, a), spec.n_kv_heads)
+    p0 = state.k_cache.shape[0]
+    n = orc.n_candidate_blocks(p0, spec.n_init, spec.block, spec.n_local_prev)
+    sc = orc.block_scores(pkv, table[:, :n])
+    c = min(spec.k_blocks, n)
+    picks = [orc.select_blocks(sc[g], c) for g in range(spec.n_kv_heads)]
+    set_diffs = sum(len(set(gpu["sel"][g][:gpu["c"]].tolist()) ^ set(picks[g][0].tolist())) for g in range(spec.n_kv_heads))
+    G = spec.group
+    o, _ = orc.retrieval_attention(q[:, head * G:(head + 1) * G], k[:, head:head + 1], v[:, head:head + 1],
+                                   state.k_cache[:, head:head + 1], state.v_cache[:, head:head + 1], p0,
+                                   [gpu["sel"][head][:gpu["c"]]], spec.n_init, spec.block, spec.n_local_prev)
+    d = np.abs(gpu["out"][:, head * G:(head + 1) * G].astype(np.float64) - o)
+    return {"max_abs": float(d.max()), "mean_abs": float(d.mean()), "count_matches": bool(gpu["c"] == c),
+            "selected_set_differences": int(set_diffs), "out_dtype": "bf16",
+            "sample": f"attention output of the {G} query heads of KV head {head} at the last window (all {spec.window} tokens), "
+                      f"block sets of all {spec.n_kv_heads} KV heads"}
+
+
+def cpu_baseline(spec, budget_s=12.0, gpu=None):
     """The oracle as it stands on the host cores: whole windows (steps 1-4 and the attention of all
-    KV heads) repeated until about `budget_s` seconds of work have been timed."""
+    KV heads) repeated until about `budget_s` seconds of work have been timed.  Returns the baseline
+    record and, when a device result is given, its comparison with the oracle."""
     import torch
     st, q, k, v = _oracle_state(spec)
+    parity = oracle_parity(spec, st, q, k, v, gpu) if gpu is not None else None
     heads = list(range(spec.n_kv_heads))
     _oracle_sample(spec, st, q, k, v, heads=heads[:1])        # page in BLAS
     times = []
@@ -426,10 +574,22 @@ def cpu_baseline(spec, budget_s=12.0):
         t14, tatt = _oracle_sample(spec, st, q, k, v, heads=heads)
         times.append(t14 + tatt)
     est = float(np.mean(times))
-    cores = int(os.environ.get("OMP_NUM_THREADS", 0)) or torch.get_num_threads()
-    return {"value": spec.window / est, "unit": UNIT, "cores": cores, "kind": "oracle",
+    return {"value": spec.window / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "sample": f"{len(times)} whole windows of the bench workload (steps 1-4 + attention of all "
-                      f"{spec.n_kv_heads} KV heads), {sum(times):.1f} s of oracle time, mean {est:.3f} s per window"}
+                      f"{spec.n_kv_heads} KV heads), {sum(times):.1f} s of oracle time, mean {est:.3f} s per window; "
+                      "NumPy fp64, its matrix products on the BLAS thread pool"}, parity
+
+
+def blas_threads() -> int:
+    """Threads the oracle's matrix products actually use: the size of NumPy's BLAS pool."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return int(os.environ.get("OMP_NUM_THREADS", 0)) or (os.cpu_count() or 1)
 
 
 def run_reference(args):
@@ -446,9 +606,8 @@ def run_reference(args):
         if i >= args.warmup:
             times.append(t14 + tatt)
     ms = 1e3 * float(np.mean(times))
-    import torch
     val = spec.window / (ms * 1e-3)
-    cores = torch.get_num_threads()
+    cores = blas_threads()
     sample = "each step: one whole window of the bench workload through the oracle (steps 1-4 + attention of all 8 KV heads)"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
@@ -480,18 +639,16 @@ def _time_stage(fn, iters, flush):
         evs.append((e0, e1))
     torch.cuda.synchronize()
     t = sorted(a.elapsed_time(b) for a, b in evs)
-    return 1e3 * t[len(t) // 2]          # median, microseconds
+    return 1e3 * t[len(t) // 2], 1e3 * t[0]          # median and minimum, microseconds
 
 
-def run_stack32(args):
+def measure_stack32(iters, dev):
     """All 32 layers of the LLaMA3-8B shape batched in one launch per stage at the last window of a
     32k prefill: Q = 134 MB, representative table = 66 MB per launch (larger than or comparable
     to L2; L2 is flushed before every timed launch)."""
     import torch
     from paper_2502_13542_b200 import binding as B
     from paper_2502_13542_b200 import workloads as wl
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
     spec = wl.llama3_8b_stack32()
     L = spec.n_layers
     cfg = B.make_config(spec, out_dtype=B.BF16)
@@ -531,22 +688,22 @@ def run_stack32(args):
     for name, (fn, nbytes) in stages.items():
         for _ in range(3):
             fn()
-        us = _time_stage(fn, args.steps if args.steps < 100 else 30, flush)
-        res[name] = {"us": us, "bytes": nbytes, "GBps": nbytes / us / 1e3, "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+        us, us_min = _time_stage(fn, iters, flush)
+        res[name] = {"us": us, "min_us": us_min, "bytes": nbytes, "GBps": nbytes / us / 1e3,
+                     "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
     assert int(st.status.item()) == 0
-    print(json.dumps({"workload": "llama3_8b_stack32_32k: 32 layers batched per launch, last window", "stages": res,
-                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cold_l2": "512 MB read through L2 before every timed launch"}))
+    return {"workload": "llama3_8b_stack32_32k: 32 layers batched per launch, last window", "stages": res,
+            "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "cold_l2": "512 MB read through L2 before every timed launch"}
 
 
-def run_decode16(args):
+def measure_decode16(iters, dev, decode_splits=1):
     """Decode, 16 sequences with contexts ~ U[32768, 131072], one token per step, one layer per
     launch, probes fixed: score + cut-off/select over every sequence's table, then the decode
     attention over [128 initial | 32 selected blocks | >= 512 local] keys per KV head."""
     import torch
     from paper_2502_13542_b200 import binding as B
     from paper_2502_13542_b200 import workloads as wl
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
     spec = wl.decode_batch16().replace(n_layers=1, cap_blocks=32)
     S = spec.n_seq
     ctx = (wl.decode_contexts(spec) // spec.window) * spec.window
@@ -595,8 +752,8 @@ def run_decode16(args):
                        st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
 
     ws = None
-    if args.decode_splits > 1:           # split form of the decode kernel, with a caller-owned workspace
-        ws = torch.zeros(B.decode_workspace_bytes(cfg, states[0].batch, 1, args.decode_splits), dtype=torch.uint8, device=dev)
+    if decode_splits > 1:           # split form of the decode kernel, with a caller-owned workspace
+        ws = torch.zeros(B.decode_workspace_bytes(cfg, states[0].batch, 1, decode_splits), dtype=torch.uint8, device=dev)
 
     def attention():
         st = cur()
@@ -605,7 +762,7 @@ def run_decode16(args):
                                   st.sel_count, out, None, st.status)
         else:
             B.decode_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
-                               st.sel_count, out, None, args.decode_splits, ws, st.status)
+                               st.sel_count, out, None, decode_splits, ws, st.status)
         it["i"] += 1
     e = 2
     n_blocks = [wl.n_candidates(spec, int(c)) for c in ctx]
@@ -618,7 +775,6 @@ def run_decode16(args):
     att_bytes = sum(kk * spec.n_kv_heads * spec.head_dim * e * 2 for kk in keys)
     peaks = load_peaks()
     res = {}
-    iters = args.steps if args.steps < 100 else 30
     def score_only():
         st = cur()
         B.score_blocks(cfg, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, st.scores, st.theta, st.status)
@@ -632,12 +788,106 @@ def run_decode16(args):
                              ("score_blocks", score_only, score_bytes), ("select_cutoff", select_only, 0)):
         for _ in range(3):
             fn()
-        us = _time_stage(fn, iters, flush)
-        res[name] = {"us": us, "bytes": nbytes, "GBps": nbytes / us / 1e3, "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+        us, us_min = _time_stage(fn, iters, flush)
+        res[name] = {"us": us, "min_us": us_min, "bytes": nbytes, "GBps": nbytes / us / 1e3,
+                     "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
     assert all(int(st.status.item()) == 0 for st in states)
-    print(json.dumps({"workload": f"decode16: 16 sequences, contexts {int(ctx.min())}..{int(ctx.max())}, 1 token per step, one layer per launch, {n_pools} layer pools rotated",
-                      "keys_per_head": {"min": min(keys), "max": max(keys)}, "stages": res,
-                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cold_l2": "512 MB read through L2 before every timed launch"}))
+    return {"workload": f"decode16: 16 sequences, contexts {int(ctx.min())}..{int(ctx.max())}, 1 token per step, "
+                        f"one layer per launch, {n_pools} layer pools rotated",
+            "keys_per_head": {"min": min(keys), "max": max(keys)}, "stages": res,
+            "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "cold_l2": "512 MB read through L2 before every timed launch"}
+
+
+def measure_score_full(iters, dev):
+    """Step 3 at the size of a whole decode step: 16 sequences x 32 layers scored in ONE launch, as
+    Algorithm 1 does when every layer's scores are taken before any budget.  The table holds
+    contexts ~ U[32768, 131072] (n = 251..1019 candidate blocks per sequence), filled with seeded
+    random keys and their true inverse norms (the kernel's traffic does not depend on the values);
+    algorithmic bytes = the candidate rows, their inverse norms and the scores written."""
+    import torch
+    from paper_2502_13542_b200 import binding as B
+    from paper_2502_13542_b200 import workloads as wl
+    spec = wl.decode_batch16()
+    S, L, Hkv, D, r = spec.n_seq, spec.n_layers, spec.n_kv_heads, spec.head_dim, spec.n_repr
+    ctx = (wl.decode_contexts(spec) // spec.window) * spec.window
+    n_blocks = [wl.n_candidates(spec, int(c)) for c in ctx]
+    n_cap = max(n_blocks)
+    cfg = B.make_config(spec, out_dtype=B.BF16, n_cap=n_cap, max_context=int(ctx.max()) + spec.window)
+    gen = torch.Generator(device=dev).manual_seed(spec.seed)
+    U = S * L
+    repr_k = torch.empty(U, Hkv, n_cap, r, D, dtype=torch.bfloat16, device=dev)
+    inv = torch.empty(U, Hkv, n_cap, r, dtype=torch.float32, device=dev)
+    for u0 in range(0, U, 32):                       # filled in slices: the fp32 temporaries stay small
+        x = torch.randn(32, Hkv, n_cap, r, D, device=dev, generator=gen)
+        repr_k[u0:u0 + 32] = x.to(torch.bfloat16)
+        inv[u0:u0 + 32] = 1.0 / repr_k[u0:u0 + 32].float().norm(dim=-1)
+        del x
+    probe = torch.randn(U, Hkv, D, device=dev, generator=gen)
+    scores = torch.zeros(U, Hkv, n_cap, device=dev)
+    theta = torch.zeros(U, Hkv, device=dev)
+    n_cand = torch.tensor(n_blocks, dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    batch = B.Batch(S, L, 0)
+    nbytes = L * sum(n * Hkv * r * (D * 2 + 4) + n * Hkv * 4 for n in n_blocks)
+    fn = lambda: B.score_blocks(cfg, batch, probe, repr_k, inv, n_cand, scores, theta, status)
+    for _ in range(3):
+        fn()
+    flush = l2_flusher(dev)
+    us, us_min = _time_stage(fn, iters, flush)
+    assert int(status.item()) == 0
+    peaks = load_peaks()
+    return {"workload": f"score_blocks over 16 sequences x 32 layers in one launch ({nbytes / 1e9:.2f} GB of table rows)",
+            "us": us, "min_us": us_min, "bytes": nbytes, "GBps": nbytes / us / 1e3,
+            "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+
+
+def measure_long131k(dev, peaks):
+    """The 131072-token prefill of one layer (k = cap = 128 blocks): every one of the 256 windows is
+    timed as it is prefilled (L2 flushed before each), which gives the sweep average
+    131072 / sum_t t_window(t); the last window (17,024 keys per query) is then repeated for the
+    step time and the attention's tensor-core fraction at that length."""
+    import torch
+    from paper_2502_13542_b200 import binding as B
+    from paper_2502_13542_b200 import workloads as wl
+    spec = wl.long_131k()
+    flush = l2_flusher(dev)
+    sweep = []
+    cfg, states, inputs = build_states(spec, 1, dev, sweep_times=sweep, flush=flush)
+    st = states[0]
+    q, k, v, out = inputs[0]
+    W = spec.window
+    p0 = (spec.n_windows - 1) * W
+    att, step = [], []
+    for i in range(23):
+        flush()
+        e0, e1, e2, e3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+        e0.record()
+        st.step(q, k, v, out, advance=False, overlap_append=True)
+        e1.record()
+        flush()
+        e2.record()
+        B.retrieval_attention(cfg, st.batch, q, k, v, W, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                              st.sel_count, out, None, st.status)
+        e3.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            step.append(1e3 * e0.elapsed_time(e1)); att.append(1e3 * e2.elapsed_time(e3))
+    assert int(st.status.item()) == 0
+    sweep.append(float(np.median(step)))               # the last window, which the prefill loop leaves out
+    c_sel = int(st.sel_count.item())
+    flops = attention_flops(spec, p0, c_sel)
+    att_us = float(np.median(att))
+    tf = flops / (att_us * 1e-6) / 1e12
+    return {"workload": "llama3_8b_layer_131k: 256 windows of 512 tokens, k = cap = 128 blocks",
+            "last_window": {"step_us": float(np.median(step)), "step_min_us": float(np.min(step)),
+                            "tokens_per_s_layer": W / (float(np.median(step)) * 1e-6), "selected_blocks": c_sel,
+                            "attention_us": att_us, "attention_min_us": float(np.min(att)),
+                            "attention_TFLOPs": tf, "attention_frac_of_measured_bf16": tf / peaks["bf16_tflops"],
+                            "attention_flops": flops},
+            "sweep": {"windows": len(sweep), "sum_ms": float(np.sum(sweep)) * 1e-3,
+                      "tokens_per_s_layer": spec.context / (float(np.sum(sweep)) * 1e-6),
+                      "first_window_us": sweep[0], "window_64_us": sweep[63], "window_128_us": sweep[127]}}
 
 
 def main():
@@ -649,24 +899,46 @@ def main():
     ap.add_argument("--copies", type=int, default=8)
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="layer32k", choices=["layer32k", "stack32", "decode16"],
-                    help="layer32k = the headline line; the others print per-stage HBM figures on batched shapes")
+    ap.add_argument("--workload", default="layer32k", choices=["layer32k", "stack32", "decode16", "long131k", "scorefull"],
+                    help="layer32k = the headline line (which also carries the others' figures unless --headline-only); "
+                         "the others print one secondary measurement alone")
+    ap.add_argument("--reps", type=int, default=20, help="repetitions of the timed K-step region (median reported)")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the secondary measurements (batched stages, 131k sweep, sustained loop)")
     ap.add_argument("--decode-splits", type=int, default=1,
                     help="decode16 workload: key-stream splits per (sequence, KV head) of the decode attention")
     ap.add_argument("--profile-region", action="store_true",
                     help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world:
+        if "WORLD_SIZE" in os.environ or args.gpus < 1:
+            sys.exit(f"bench.py: --gpus {args.gpus} does not match WORLD_SIZE={world} of the launcher")
+        # started as a plain process with --gpus N > 1: become N ranks, one per GPU, under torchrun
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", os.environ.get("MASTER_PORT", "29517"),
+               os.path.abspath(__file__)] + sys.argv[1:]
+        os.execv(sys.executable, cmd)
     if args.impl == "reference":
         args.steps = min(args.steps, 30)
         args.warmup = min(args.warmup, 2)
         run_reference(args)
-    elif args.workload == "stack32":
-        run_stack32(args)
-    elif args.workload == "decode16":
-        run_decode16(args)
-    else:
+    elif args.workload == "layer32k":
         run_ours(args)
+    else:
+        import torch
+        torch.cuda.set_device(0)
+        dev = torch.device("cuda", 0)
+        iters = args.steps if args.steps < 100 else 30
+        if args.workload == "stack32":
+            print(json.dumps(measure_stack32(iters, dev)))
+        elif args.workload == "decode16":
+            print(json.dumps(measure_decode16(iters, dev, args.decode_splits)))
+        elif args.workload == "scorefull":
+            print(json.dumps(measure_score_full(iters, dev)))
+        else:
+            print(json.dumps(measure_long131k(dev, load_peaks())))
 
 
 if __name__ == "__main__":

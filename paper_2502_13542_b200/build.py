@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libactqkv.so")
-SOURCES = ["api.cu", "bias_probe.cu", "score.cu", "select.cu", "attention_simt.cu", "attention_tc.cu", "attention_tc2.cu", "attention_decode.cu", "append.cu"]
+SOURCES = ["api.cu", "bias_probe.cu", "score.cu", "select.cu", "attention_simt.cu", "attention_tc.cu", "attention_tc2.cu", "attention_tc4.cu", "attention_decode.cu", "append.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static", "-Wno-deprecated-gpu-targets"]
 

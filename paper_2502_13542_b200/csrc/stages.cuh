@@ -49,6 +49,10 @@ int launch_attention_tc(const actqkv_config* cfg, const Batch& b, const AttnArgs
 // The same kernel for pairs of CTAs sharing each K / V tile (needs an even number of query heads per KV head).
 bool attention_tc2_supported(const actqkv_config* cfg, int n_tokens);
 int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
+// Four query heads of a KV group per CTA pair, the key stream split over the two pairs of a 4-CTA
+// cluster (needs a multiple of 4 query heads per KV head).
+bool attention_tc4_supported(const actqkv_config* cfg, int n_tokens);
+int launch_attention_tc4(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 
 // Short steps (decode): one CTA per (unit, KV head, split of the key stream), G query heads packed
 // in the M tile; n_splits > 1 needs a workspace of attention_decode_workspace_bytes().

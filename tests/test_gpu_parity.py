@@ -297,11 +297,11 @@ def test_edge_cases_and_errors(B):
     assert int(st4.status.item()) == 0
 
 
-@pytest.mark.parametrize("kernel", ["pair", "tc1"])
+@pytest.mark.parametrize("kernel", ["cluster4", "pair", "tc1"])
 @pytest.mark.parametrize("target", [1, 3])
 def test_tc_attention_repeatable_and_matches_general_kernel(B, target, kernel):
-    """The tensor-core attention (the CTA-pair kernel the shape selects by default, and the
-    single-CTA kernel) is run many times on the same state: every run must give the same bits
+    """The tensor-core attention (the 4-CTA-cluster kernel the shape selects by default, the
+    CTA-pair kernel and the single-CTA kernel) is run many times on the same state: every run must give the same bits
     (no timing dependence), and agree with the general fp32 kernel.  Window 1 gives the shortest
     key-tile loops (5 to 8 tiles), window 3 longer ones."""
     import torch
@@ -328,7 +328,7 @@ def test_tc_attention_repeatable_and_matches_general_kernel(B, target, kernel):
     gen = torch.zeros_like(out)
     attend(gen, B.ATTN_GENERAL)
     torch.cuda.synchronize()
-    which = B.ATTN_SINGLE_CTA if kernel == "tc1" else B.ATTN_AUTO
+    which = {"tc1": B.ATTN_SINGLE_CTA, "pair": B.ATTN_PAIR, "cluster4": B.ATTN_AUTO}[kernel]
     outs = [torch.zeros_like(out) for _ in range(8)]
     ref = None
     for rep in range(60):
@@ -338,10 +338,10 @@ def test_tc_attention_repeatable_and_matches_general_kernel(B, target, kernel):
         if ref is None:
             ref = outs[0].clone()
             # The single-CTA kernel rounds P to bf16 as a high and a low part (16 bits in all); the
-            # pair kernel rounds P to fp16 (relative error 2^-12), which the largest value channels
+            # pair and cluster kernels round P to fp16 (relative error 2^-12), which the largest value channels
             # of this workload (|v| up to about 40) turn into at most 40 * 2^-12 = 1e-2 absolute.
             d = (gen - ref).abs()
-            assert d.max().item() < (1e-2 if kernel == "pair" else 2e-3)
+            assert d.max().item() < (2e-3 if kernel == "tc1" else 1e-2)
             assert d.mean().item() < 2e-4
         for o in outs:
             assert torch.equal(o, ref), f"run {rep}: tensor-core attention not repeatable"
