@@ -96,10 +96,11 @@ enum { ACTQKV_THETABAR_STREAMING = 0, ACTQKV_THETABAR_ALG1 = 1 };
  * compares against (Sec. 1; the "w/o APQ" row of its ablation, Sec. 5.3). */
 enum { ACTQKV_PROBE_ACTIVATION = 0, ACTQKV_PROBE_MEAN_POOL = 1 };
 /* Which kernel serves actqkv_retrieval_attention: chosen by shape (default); the general
- * fp32-accumulate kernel; the single-CTA tensor-core kernel; the two-head CTA-pair kernel.  The
- * last three exist for testing one kernel against another; results agree within the rounding of
- * the products. */
-enum { ACTQKV_ATTN_AUTO = 0, ACTQKV_ATTN_GENERAL = 1, ACTQKV_ATTN_SINGLE_CTA = 2, ACTQKV_ATTN_PAIR = 3 };
+ * fp32-accumulate kernel; the single-CTA tensor-core kernel; the 4-CTA-cluster kernel that serves
+ * four query heads per KV-head tile (G a multiple of 4; measured slower than the default CTA-pair
+ * kernel, kept for comparison).  The non-default values exist for testing one kernel against
+ * another; results agree within the rounding of the products. */
+enum { ACTQKV_ATTN_AUTO = 0, ACTQKV_ATTN_GENERAL = 1, ACTQKV_ATTN_SINGLE_CTA = 2, ACTQKV_ATTN_CLUSTER4 = 3 };
 
 /* Host POD describing the model / cache geometry.  Passed by const pointer (host). */
 typedef struct actqkv_config {
@@ -229,8 +230,7 @@ int actqkv_score_select(const actqkv_config* cfg, const actqkv_batch* batch, con
  *   out          [U][n_tokens][Hq][D]   cfg->out_dtype out
  *   lse          [U][Hq][n_tokens]      fp32 out, may be NULL (natural-log sum of exp)
  * bf16, D = 128, 16-token pages: steps whose n_tokens is a multiple of 128 run on the tcgen05
- * prefill kernels (4-CTA clusters serving four query heads per KV-head tile when G is a multiple
- * of 4, CTA pairs when G is even), steps of n_tokens <= 128 / G tokens on the tcgen05
+ * prefill kernels (CTA pairs when G is even), steps of n_tokens <= 128 / G tokens on the tcgen05
  * decode kernel (one CTA per KV head; see actqkv_decode_attention for the split form); every
  * other shape runs on the general fp32-accumulate kernel.
  * Preconditions of the tcgen05 kernels (the general kernel has none of them):

@@ -27,7 +27,7 @@ REPR_CHUNK_MEAN, REPR_STRIDED_TOKEN = 0, 1
 AGG_MEAN, AGG_MAX = 0, 1
 THETABAR_STREAMING, THETABAR_ALG1 = 0, 1
 PROBE_ACTIVATION, PROBE_MEAN_POOL = 0, 1
-ATTN_AUTO, ATTN_GENERAL, ATTN_SINGLE_CTA, ATTN_PAIR = 0, 1, 2, 3
+ATTN_AUTO, ATTN_GENERAL, ATTN_SINGLE_CTA, ATTN_CLUSTER4 = 0, 1, 2, 3
 
 DEV_BAD_PAGE, DEV_NCAND_CLAMPED, DEV_BAD_PROBE, DEV_BAD_SELECTION, DEV_TIMEOUT, DEV_TABLE_FULL = \
     1, 2, 4, 8, 16, 32

@@ -55,8 +55,8 @@ extern "C" int actqkv_retrieval_attention(const actqkv_config* cfg, const actqkv
   // cfg->attention_kernel pins one kernel (for comparing kernels with each other); 0 picks by shape
   const bool simt_only = cfg->attention_kernel == ACTQKV_ATTN_GENERAL;
   const bool tc1_only = cfg->attention_kernel == ACTQKV_ATTN_SINGLE_CTA;
-  const bool pair_only = cfg->attention_kernel == ACTQKV_ATTN_PAIR;
-  if (!simt_only && !tc1_only && !pair_only && attention_tc4_supported(cfg, n_tokens)) return launch_attention_tc4(cfg, b, a, st);
+  if (cfg->attention_kernel == ACTQKV_ATTN_CLUSTER4 && attention_tc4_supported(cfg, n_tokens))
+    return launch_attention_tc4(cfg, b, a, st);
   if (!simt_only && !tc1_only && attention_tc2_supported(cfg, n_tokens)) return launch_attention_tc2(cfg, b, a, st);
   if (!simt_only && attention_tc_supported(cfg, n_tokens)) return launch_attention_tc(cfg, b, a, st);
   if (!simt_only && attention_decode_supported(cfg, n_tokens)) return launch_attention_decode(cfg, b, a, 1, nullptr, st);

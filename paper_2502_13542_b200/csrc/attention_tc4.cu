@@ -15,23 +15,31 @@
 //     distributed shared memory and finishes the other set: pair 0 writes set X, pair 1 set Y.
 //     No workspace in global memory, no second kernel, and 8 x 4 units fill 128 SMs.
 //
-// Roles per CTA (512 threads = 4 warpgroups; registers are moved between them with setmaxnreg):
+// Roles per CTA (512 threads):
 //   warp 0      K producer (TMA page gather) and the Q tiles
-//   warp 1      MMA issuer (leader CTA of the pair only): ONE thread issues every product, in
-//               order:  ... PV_X(j)  QK_X(j+1)  PV_Y(j)  QK_Y(j+1) ...  The tensor pipe executes in
-//               issue order, so QK_X(j+1) overwrites S_X only after PV_X(j) has read P_X from it,
-//               and while the pipe works on set Y the softmax of set X runs (and the reverse).
+//   warps 1, 3  MMA issuers (leader CTA of the pair only), one thread each: warp 1 issues the
+//               products of set X, warp 3 those of set Y, each in order.  A key tile is handled as
+//               two BLOCKS of 64 keys; block b of a set uses S buffer b % 2:
+//                   ... PV(b)  QK(b+2)  PV(b+1)  QK(b+3) ...
+//               The tensor pipe executes one thread's products in issue order, so QK(b+2) overwrites
+//               its S buffer only after PV(b) has read P(b) from it, and while a softmax thread works
+//               on block b the scores of block b + 1 are already waiting for it.  A ring slot is
+//               released when both issuers have committed their last product on it.
 //   warp 2      V producer
-//   warps 4-7   softmax of set X, one thread per query row (128 fp32 scores in registers: no
-//               shuffles for the row maximum or sum)
-//   warps 8-11  softmax of set Y.  Every scheduler of the SM holds one warp of each set; their
-//               phases alternate, so one set's exponentials fill the special-function unit while
-//               the other set waits, loads and takes maxima.
+//   warps 4-7   softmax of set X, one thread per query row (a block's 64 fp32 scores in registers:
+//               no shuffles for the row maximum or sum)
+//   warps 8-11  softmax of set Y.  Every scheduler of the SM holds one warp of each set.
 //   warps 12-15 V conversion (bf16 -> fp16 in place, two tiles ahead) and O correction
-// P is fp16 (11 significant bits) and overwrites the first 64 columns of its S buffer; the running
+// P is fp16 (11 significant bits) and overwrites the first 32 columns of its S buffer; the running
 // maximum used for P may lag the true one by up to 2^8 (fp16 range), and when it moves O is
 // rescaled by the correction warps, off the softmax threads' path.
-// TMEM columns (every CTA): S_X [0,128)  S_Y [128,256)  O_X [256,384)  O_Y [384,512).
+// TMEM columns (every CTA): S_X [0,64) [64,128)  S_Y [128,192) [192,256)  O_X [256,384)  O_Y [384,512).
+// Measured on the LLaMA3-8B layer at 32k context: 60.8 us per call against 55.8 us for the two-head
+// pair kernel, so the dispatcher takes this kernel only when asked to (ACTQKV_ATTN_CLUSTER4).  A
+// tcgen05.mma of M = 256 occupies the tensor pipe ~62 cycles for every N <= 128, so the 64-key
+// blocks that double-buffered S needs (TMEM has 512 columns: two sets x (2 x 64 S + 128 O)) spend
+// twice the pipe time on Q K^T; with 128-key blocks and one S buffer per set the pipe waits for the
+// softmax -> P -> P V -> Q K^T chain instead (4,350 cycles per key tile measured).
 // No TMA multicast anywhere.  Every wait on an mbarrier is bounded; on expiry the CTA flags
 // ACTQKV_DEV_TIMEOUT, stops issuing work and drains; every CTA of the cluster always reaches the
 // cluster barriers of the hand-over, so nobody waits for a CTA that gave up.
@@ -54,9 +62,10 @@ constexpr uint32_t kHalfBytes = 16 * 1024;               // what one CTA holds o
 constexpr uint32_t kKSubBytes = 64 * 128;                // [64 keys x 64 channels] sub-tile of a K half
 constexpr uint32_t kQBytes = 2 * kTileBytes;             // the Q tiles of sets X and Y
 constexpr uint32_t kSmemTiles = kQBytes + (kRingK + kRingV) * kHalfBytes;
-constexpr int kNumBars = 1 + 2 * kRingK + 3 * kRingV + 5 * 2 + 1;
-constexpr uint32_t kBarBytes = 320;                      // barriers, TMEM slot, abort flag
-constexpr uint32_t kXchgBytes = (2 + 2) * 128 * 4;       // O factors [set][row]; hand-over of (maximum, sum) [2][row]
+constexpr int kBlk = 64;                                 // keys per block = columns of an S buffer
+constexpr int kNumBars = 1 + 2 * kRingK + 3 * kRingV + 4 * 4 + 2 + 1;
+constexpr uint32_t kBarBytes = 384;                      // barriers, TMEM slot, abort flag
+constexpr uint32_t kXchgBytes = 4 * 128 * 4;             // O factors [set][buffer][row]; reused for the hand-over of (maximum, sum) [row][2]
 constexpr uint32_t kSmemNeeded = kSmemTiles + kBarBytes + kXchgBytes;
 constexpr uint32_t kSmemBytes = 227 * 1024;              // everything an SM offers one CTA
 constexpr uint32_t kStageBytes = 128 * 128 * 4;          // one set's partial O in fp32, staged over the rings
@@ -125,90 +134,6 @@ __device__ __forceinline__ void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint32
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// Registers move between the warpgroups: the softmax threads hold a whole row of scores.
-template <int kRegs> __device__ __forceinline__ void reg_release() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs)); }
-template <int kRegs> __device__ __forceinline__ void reg_acquire() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs)); }
-constexpr int kRegsProducer = 48, kRegsSoftmax = 192, kRegsCorrection = 80;
-static_assert(128 * (kRegsProducer + 2 * kRegsSoftmax + kRegsCorrection) <= 65536, "register file");
-
-// One query row: 128 fp32 columns as 64 packed pairs (column 2i in the low half of r[i]); the wait
-// is part of the same statement, so no consumer can be scheduled ahead of it.
-#define TMEM_LD128P_WAIT(taddr, r) \
-  asm volatile( \
-      "{\n\t.reg .b32 t<128>;\n\t" \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t0,t1,t2,t3,t4,t5,t6,t7,t8,t9,t10,t11,t12,t13,t14,t15,t16,t17,t18,t19,t20,t21,t22,t23,t24,t25,t26,t27,t28,t29,t30,t31}, [%64];\n\t" \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t32,t33,t34,t35,t36,t37,t38,t39,t40,t41,t42,t43,t44,t45,t46,t47,t48,t49,t50,t51,t52,t53,t54,t55,t56,t57,t58,t59,t60,t61,t62,t63}, [%65];\n\t" \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t64,t65,t66,t67,t68,t69,t70,t71,t72,t73,t74,t75,t76,t77,t78,t79,t80,t81,t82,t83,t84,t85,t86,t87,t88,t89,t90,t91,t92,t93,t94,t95}, [%66];\n\t" \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {t96,t97,t98,t99,t100,t101,t102,t103,t104,t105,t106,t107,t108,t109,t110,t111,t112,t113,t114,t115,t116,t117,t118,t119,t120,t121,t122,t123,t124,t125,t126,t127}, [%67];\n\t" \
-      "tcgen05.wait::ld.sync.aligned;\n\t" \
-      "mov.b64 %0, {t0, t1};\n\t" \
-      "mov.b64 %1, {t2, t3};\n\t" \
-      "mov.b64 %2, {t4, t5};\n\t" \
-      "mov.b64 %3, {t6, t7};\n\t" \
-      "mov.b64 %4, {t8, t9};\n\t" \
-      "mov.b64 %5, {t10, t11};\n\t" \
-      "mov.b64 %6, {t12, t13};\n\t" \
-      "mov.b64 %7, {t14, t15};\n\t" \
-      "mov.b64 %8, {t16, t17};\n\t" \
-      "mov.b64 %9, {t18, t19};\n\t" \
-      "mov.b64 %10, {t20, t21};\n\t" \
-      "mov.b64 %11, {t22, t23};\n\t" \
-      "mov.b64 %12, {t24, t25};\n\t" \
-      "mov.b64 %13, {t26, t27};\n\t" \
-      "mov.b64 %14, {t28, t29};\n\t" \
-      "mov.b64 %15, {t30, t31};\n\t" \
-      "mov.b64 %16, {t32, t33};\n\t" \
-      "mov.b64 %17, {t34, t35};\n\t" \
-      "mov.b64 %18, {t36, t37};\n\t" \
-      "mov.b64 %19, {t38, t39};\n\t" \
-      "mov.b64 %20, {t40, t41};\n\t" \
-      "mov.b64 %21, {t42, t43};\n\t" \
-      "mov.b64 %22, {t44, t45};\n\t" \
-      "mov.b64 %23, {t46, t47};\n\t" \
-      "mov.b64 %24, {t48, t49};\n\t" \
-      "mov.b64 %25, {t50, t51};\n\t" \
-      "mov.b64 %26, {t52, t53};\n\t" \
-      "mov.b64 %27, {t54, t55};\n\t" \
-      "mov.b64 %28, {t56, t57};\n\t" \
-      "mov.b64 %29, {t58, t59};\n\t" \
-      "mov.b64 %30, {t60, t61};\n\t" \
-      "mov.b64 %31, {t62, t63};\n\t" \
-      "mov.b64 %32, {t64, t65};\n\t" \
-      "mov.b64 %33, {t66, t67};\n\t" \
-      "mov.b64 %34, {t68, t69};\n\t" \
-      "mov.b64 %35, {t70, t71};\n\t" \
-      "mov.b64 %36, {t72, t73};\n\t" \
-      "mov.b64 %37, {t74, t75};\n\t" \
-      "mov.b64 %38, {t76, t77};\n\t" \
-      "mov.b64 %39, {t78, t79};\n\t" \
-      "mov.b64 %40, {t80, t81};\n\t" \
-      "mov.b64 %41, {t82, t83};\n\t" \
-      "mov.b64 %42, {t84, t85};\n\t" \
-      "mov.b64 %43, {t86, t87};\n\t" \
-      "mov.b64 %44, {t88, t89};\n\t" \
-      "mov.b64 %45, {t90, t91};\n\t" \
-      "mov.b64 %46, {t92, t93};\n\t" \
-      "mov.b64 %47, {t94, t95};\n\t" \
-      "mov.b64 %48, {t96, t97};\n\t" \
-      "mov.b64 %49, {t98, t99};\n\t" \
-      "mov.b64 %50, {t100, t101};\n\t" \
-      "mov.b64 %51, {t102, t103};\n\t" \
-      "mov.b64 %52, {t104, t105};\n\t" \
-      "mov.b64 %53, {t106, t107};\n\t" \
-      "mov.b64 %54, {t108, t109};\n\t" \
-      "mov.b64 %55, {t110, t111};\n\t" \
-      "mov.b64 %56, {t112, t113};\n\t" \
-      "mov.b64 %57, {t114, t115};\n\t" \
-      "mov.b64 %58, {t116, t117};\n\t" \
-      "mov.b64 %59, {t118, t119};\n\t" \
-      "mov.b64 %60, {t120, t121};\n\t" \
-      "mov.b64 %61, {t122, t123};\n\t" \
-      "mov.b64 %62, {t124, t125};\n\t" \
-      "mov.b64 %63, {t126, t127};\n\t" \
-      "}" \
-      : "=l"(r[0]), "=l"(r[1]), "=l"(r[2]), "=l"(r[3]), "=l"(r[4]), "=l"(r[5]), "=l"(r[6]), "=l"(r[7]), "=l"(r[8]), "=l"(r[9]), "=l"(r[10]), "=l"(r[11]), "=l"(r[12]), "=l"(r[13]), "=l"(r[14]), "=l"(r[15]), "=l"(r[16]), "=l"(r[17]), "=l"(r[18]), "=l"(r[19]), "=l"(r[20]), "=l"(r[21]), "=l"(r[22]), "=l"(r[23]), "=l"(r[24]), "=l"(r[25]), "=l"(r[26]), "=l"(r[27]), "=l"(r[28]), "=l"(r[29]), "=l"(r[30]), "=l"(r[31]), "=l"(r[32]), "=l"(r[33]), "=l"(r[34]), "=l"(r[35]), "=l"(r[36]), "=l"(r[37]), "=l"(r[38]), "=l"(r[39]), "=l"(r[40]), "=l"(r[41]), "=l"(r[42]), "=l"(r[43]), "=l"(r[44]), "=l"(r[45]), "=l"(r[46]), "=l"(r[47]), "=l"(r[48]), "=l"(r[49]), "=l"(r[50]), "=l"(r[51]), "=l"(r[52]), "=l"(r[53]), "=l"(r[54]), "=l"(r[55]), "=l"(r[56]), "=l"(r[57]), "=l"(r[58]), "=l"(r[59]), "=l"(r[60]), "=l"(r[61]), "=l"(r[62]), "=l"(r[63]) \
-      : "r"(taddr), "r"((taddr) + 32), "r"((taddr) + 64), "r"((taddr) + 96) \
-      : "memory")
 
 // ---------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kThreads, 1)
@@ -231,18 +156,19 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   auto bar_vempty = [&](int s) { return bars + 8u * (1 + 2 * kRingK + kRingV + s); };
   auto bar_vready = [&](int s) { return bars + 8u * (1 + 2 * kRingK + 2 * kRingV + s); };
   constexpr int kB0 = 1 + 2 * kRingK + 3 * kRingV;
-  auto bar_sfull = [&](int t) { return bars + 8u * (kB0 + t); };          // S of set t is complete
-  auto bar_pfull = [&](int t) { return bars + 8u * (kB0 + 2 + t); };      // P of set t is published (leader)
-  auto bar_pvdone = [&](int t) { return bars + 8u * (kB0 + 4 + t); };     // P V of set t has completed
-  auto bar_f = [&](int t) { return bars + 8u * (kB0 + 6 + t); };          // O factors of set t are in shared memory
-  auto bar_corr = [&](int t) { return bars + 8u * (kB0 + 8 + t); };       // O of set t is on P's maximum (leader)
+  // per (set t, S buffer u): index 2 t + u
+  auto bar_sfull = [&](int t, int u) { return bars + 8u * (kB0 + 2 * t + u); };        // S is complete
+  auto bar_pfull = [&](int t, int u) { return bars + 8u * (kB0 + 4 + 2 * t + u); };    // P is published (leader)
+  auto bar_f = [&](int t, int u) { return bars + 8u * (kB0 + 8 + 2 * t + u); };        // O factors are in shared memory
+  auto bar_corr = [&](int t, int u) { return bars + 8u * (kB0 + 12 + 2 * t + u); };    // O is on P's maximum (leader)
+  auto bar_pvdone = [&](int t) { return bars + 8u * (kB0 + 16 + t); };                 // a P V of set t has completed
   const uint32_t bar_done = bars + 8u * (kNumBars - 1);
   unsigned char* base_generic = smem_raw + (base - raw);
   unsigned char* bars_generic = base_generic + kSmemTiles;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_generic + 8 * kNumBars + 8);
-  float* f_share = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [set][128] O correction factors
-  float* ml_share = f_share + 2 * 128;                                   // [2][128] counterpart's (maximum, sum) of the set this CTA finishes
+  float* f_share = reinterpret_cast<float*>(bars_generic + kBarBytes);   // [set][buffer][128] O correction factors
+  float* ml_share = f_share;     // the factors are dead when the hand-over begins (after cluster barrier 1)                                   // [2][128] counterpart's (maximum, sum) of the set this CTA finishes
   float* stage = reinterpret_cast<float*>(base_generic + kQBytes);       // [32 column quads][128 rows][4]: counterpart's partial O
 
   const int quad = blockIdx.x >> 2, mt = blockIdx.y, unit = blockIdx.z;
@@ -260,13 +186,16 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   // ---- set-up that depends on no earlier kernel: barriers, TMEM, descriptor prefetch
   if (tid == 0) {
     mbar_init(bar_q, 1);
-    for (int s = 0; s < kRingK; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
-    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1); mbar_init(bar_vready(s), 8); }
+    for (int s = 0; s < kRingK; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 2); }
+    for (int s = 0; s < kRingV; ++s) { mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 2); mbar_init(bar_vready(s), 8); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(bar_sfull(t), 1); mbar_init(bar_pfull(t), 8); mbar_init(bar_pvdone(t), 1);
-      mbar_init(bar_f(t), 4); mbar_init(bar_corr(t), 8);
+      for (int u = 0; u < 2; ++u) {
+        mbar_init(bar_sfull(t, u), 1); mbar_init(bar_pfull(t, u), 8);
+        mbar_init(bar_f(t, u), 4); mbar_init(bar_corr(t, u), 8);
+      }
+      mbar_init(bar_pvdone(t), 1);
     }
-    mbar_init(bar_done, 1);
+    mbar_init(bar_done, 2);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -325,7 +254,6 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   bool row_ok = true;
 
   if (warp < 4) {
-    reg_release<kRegsProducer>();
     if (warp == 0 || warp == 2) {
       // =========================== TMA producers: warp 0 -> K half (and Q), warp 2 -> V half ===========================
       // This CTA's half of a tile: keys [64 r, +64) of K (all channels), channels [64 r, +64) of V
@@ -345,9 +273,11 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           tma2_load_3d(q_smem + t * kTileBytes + kSubTileBytes, &tm_q, qb, 64, h0 + t, row0);
         }
       }
-      // lanes 0-7 issue one box each.  K: (channel half, granule 4 r + slot); V: granule = lane.
+      // lanes 0-7 issue one box each.  V: granule = lane.  K: (channel half, slot); the CTA's 64
+      // key rows are [32 keys of block 0 | 32 keys of block 1], i.e. 16-key granules
+      // 2 r, 2 r + 1, 4 + 2 r, 5 + 2 r of the tile, so that block b is keys [64 b, 64 b + 64) in order.
       const int half = (lane >> 2) & 1, slot = lane & 3;
-      const int my_granule = is_v ? (lane & 7) : int(r) * 4 + slot;
+      const int my_granule = is_v ? (lane & 7) : (slot >> 1) * 4 + int(r) * 2 + (slot & 1);
       // Page lookups (sel_idx -> page_table, two dependent loads) are taken 32 granules = 4 tiles at
       // a time, one granule per lane, one chunk ahead of the tiles being issued.
       auto resolve = [&](int chunk) {
@@ -383,8 +313,9 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           const int row0 = unit * nt + (jj - past_tiles) * kBN;
           if (is_v) {
             if (lane == 0) tma_load_3d(sbase, tm_win, full, int(r) * 64, g, row0);
-          } else if (lane < 2) {
-            tma2_load_3d(sbase + lane * kKSubBytes, tm_win, full, lane * 64, g, row0 + int(r) * 64);
+          } else if (lane < 4) {        // (channel half, block): 32 keys each
+            const int hf = lane & 1, blk = lane >> 1;
+            tma2_load_3d(sbase + hf * kKSubBytes + blk * 4096u, tm_win, full, hf * 64, g, row0 + blk * kBlk + int(r) * 32);
           }
         }
         issued = j + 1;
@@ -404,73 +335,66 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           __nanosleep(200000);
         }
       }
-    } else if (warp == 1) {
-      // =========================== MMA issuer (leader CTA of the pair) ===========================
-      // One thread, one order.  Per key tile j:  PV_X(j)  QK_X(j+1)  PV_Y(j)  QK_Y(j+1).  The
+    } else if (warp == 1 || warp == 3) {
+      // =========================== MMA issuers: warp 1 set X, warp 3 set Y (leader CTA of the pair) ===========================
+      // One thread, one order.  Per 64-key block b:  PV_X(b)  QK_X(b+2)  PV_Y(b)  QK_Y(b+2).  The
       // pipe runs products in issue order, so nothing else orders the reuse of an S / P buffer.
       if (lane == 0 && leader && n_tiles > 0) {
         constexpr uint32_t kHi = desc_hi(1024u);       // descriptor high words are constants
-        constexpr uint32_t idesc_qk = make_idesc(false, 2 * kBM, kBN);
+        constexpr uint32_t idesc_qk = make_idesc(false, 2 * kBM, kBlk);
         constexpr uint32_t idesc_pv = make_idesc_f16(true, 2 * kBM, kBN);
+        const int n_blocks = 2 * n_tiles;
         bool ok = mbar_wait(bar_q, 0, abort_flag);
-        auto qk = [&](int t, int j) {
+        // S(t, b) = Q_t K(b)^T: A = this CTA's 128 query rows, B = this CTA's 32 keys of the block
+        auto qk = [&](int t, int b) {
           const uint32_t q_lo = desc_lo(q_smem + t * kTileBytes, 16u);
-          const uint32_t k_lo = desc_lo(k_ring + (j % kRingK) * kHalfBytes, 16u);
-          const uint32_t s_tmem = tmem + t * 128;
-          // A: this CTA's 128 query rows; B: this CTA's 64 keys; both advance 16 channels per step
+          const uint32_t k_lo = desc_lo(k_ring + ((b >> 1) % kRingK) * kHalfBytes + (b & 1) * 4096u, 16u);
+          const uint32_t s_tmem = tmem + t * 128 + (b & 1) * kBlk;
           mma2_ss<false>(s_tmem, q_lo, k_lo, kHi, idesc_qk);
 #pragma unroll
-          for (int k = 1; k < kD / 16; ++k) {
-            constexpr uint32_t kUnit = 16;     // descriptor addresses count 16-byte units
+          for (int k = 1; k < kD / 16; ++k) {          // both operands advance 16 channels per step
+            constexpr uint32_t kUnit = 16;             // descriptor addresses count 16-byte units
             const uint32_t a_off = ((k >> 2) * kSubTileBytes + (k & 3) * 32u) / kUnit;
             const uint32_t b_off = ((k >> 2) * kKSubBytes + (k & 3) * 32u) / kUnit;
             mma2_ss<true>(s_tmem, q_lo + a_off, k_lo + b_off, kHi, idesc_qk);
           }
         };
-        auto pv = [&](int t, int j) {
-          const uint32_t v_lo = desc_lo(v_ring + (j % kRingV) * kHalfBytes, kSubTileBytes);
-          const uint32_t p_tmem = tmem + t * 128, o_tmem = tmem + 256 + t * 128;
+        // O_t += P(t, b) V(b): A = 64 keys of P as 32 packed fp16 columns, B = this CTA's 64 channels
+        auto pv = [&](int t, int b) {
+          const uint32_t v_lo = desc_lo(v_ring + ((b >> 1) % kRingV) * kHalfBytes, kSubTileBytes) + (b & 1) * (4 * 2048u / 16u);
+          const uint32_t p_tmem = tmem + t * 128 + (b & 1) * kBlk, o_tmem = tmem + 256 + t * 128;
 #pragma unroll
-          for (int k = 0; k < kBN / 16; ++k)      // 16 keys per step: B advances 16 rows of 128 bytes, A 8 packed fp16 columns
-            mma2_ts(o_tmem, p_tmem + k * 8, v_lo + k * (2048u / 16u), kHi, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < kBlk / 16; ++k)     // 16 keys per step: B advances 16 rows of 128 bytes, A 8 packed fp16 columns
+            mma2_ts(o_tmem, p_tmem + k * 8, v_lo + k * (2048u / 16u), kHi, idesc_pv, (b > 0 || k > 0) ? 1u : 0u);
         };
+        const int t = warp == 1 ? 0 : 1;                 // this thread's set
         ok = ok && mbar_wait(bar_kfull(0), 0, abort_flag);
         if (ok) {
           tc_fence_after();
-          qk(0, 0);
-          pair_commit(bar_sfull(0), pair_mask);
-          qk(1, 0);
-          pair_commit(bar_kempty(0), pair_mask);
-          pair_commit(bar_sfull(1), pair_mask);
+          qk(t, 0); pair_commit(bar_sfull(t, 0), pair_mask);
+          qk(t, 1); pair_commit(bar_kempty(0), pair_mask); pair_commit(bar_sfull(t, 1), pair_mask);
         }
-        for (int j = 0; j < n_tiles && ok; ++j) {
-          const uint32_t ph = j & 1;
-          const bool more = j + 1 < n_tiles;
-          ok = mbar_wait(bar_vready(j % kRingV), (j / kRingV) & 1, abort_flag);   // V(j) is fp16 in both CTAs
-          ok = ok && mbar_wait(bar_corr(0), ph, abort_flag);                     // O_X is on P_X(j)'s maximum
-          ok = ok && mbar_wait(bar_pfull(0), ph, abort_flag);                    // P_X(j) published by both CTAs
+        for (int b = 0; b < n_blocks && ok; ++b) {
+          const int j = b >> 1, u = b & 1;
+          const uint32_t ph = (b >> 1) & 1;             // phase of the per-(set, buffer) barriers
+          const bool more = b + 2 < n_blocks;
+          if (u == 0) ok = mbar_wait(bar_vready(j % kRingV), (j / kRingV) & 1, abort_flag);   // V(j) is fp16 in both CTAs
+          ok = ok && mbar_wait(bar_corr(t, u), ph, abort_flag);                  // O is on P(b)'s maximum
+          ok = ok && mbar_wait(bar_pfull(t, u), ph, abort_flag);                 // P(b) published by both CTAs
           if (!ok) break;
           tc_fence_after();
-          pv(0, j);
-          pair_commit(bar_pvdone(0), pair_mask);
+          pv(t, b);
+          if (u == 1) pair_commit(bar_vempty(j % kRingV), pair_mask);
+          pair_commit(bar_pvdone(t), pair_mask);
           if (more) {
-            ok = mbar_wait(bar_kfull((j + 1) % kRingK), ((j + 1) / kRingK) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            qk(0, j + 1);
-            pair_commit(bar_sfull(0), pair_mask);
-          }
-          ok = mbar_wait(bar_corr(1), ph, abort_flag);
-          ok = ok && mbar_wait(bar_pfull(1), ph, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          pv(1, j);
-          pair_commit(bar_vempty(j % kRingV), pair_mask);
-          pair_commit(bar_pvdone(1), pair_mask);
-          if (more) {
-            qk(1, j + 1);
-            pair_commit(bar_kempty((j + 1) % kRingK), pair_mask);
-            pair_commit(bar_sfull(1), pair_mask);
+            if (u == 0) {
+              ok = mbar_wait(bar_kfull((j + 1) % kRingK), ((j + 1) / kRingK) & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            qk(t, b + 2);
+            if (u == 1) pair_commit(bar_kempty((j + 1) % kRingK), pair_mask);
+            pair_commit(bar_sfull(t, u), pair_mask);
           }
         }
         if (ok) pair_commit(bar_done, pair_mask);
@@ -482,7 +406,6 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   }
   else if (warp >= 12) {
     // =========================== V converters / O correction ===========================
-    reg_release<kRegsCorrection>();
     // This CTA's half of every V tile, as it landed (bf16), becomes fp16 in place, 128 bytes per
     // thread, kLag tiles ahead of its use; one arrival per warp on the leader's "V ready" barrier.
     const int ct = tid - 12 * 32;                         // 0..127 = this thread's query row in both sets
@@ -507,17 +430,18 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       }
       const int j = it - kLag;
       if (j >= 0) {
-        // The maxima of tile j are known: where a row's maximum grew, its O (on the old maximum) is
-        // scaled down before P(j) V(j) is added.  The softmax threads do not wait for this.
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-          ok = mbar_wait(bar_f(t), j & 1, abort_flag);
+        // The maxima of the two blocks of tile j are known: where a row's maximum grew, its O (on
+        // the old maximum) is scaled down before P V of that block is added.  The softmax threads
+        // do not wait for this.  Order as the issuer's: (block, set) = (2j, X) (2j, Y) (2j+1, X) (2j+1, Y).
+        for (int bt = 0; bt < 4 && ok; ++bt) {
+          const int u = bt >> 1, t = bt & 1, b = 2 * j + u;
+          ok = mbar_wait(bar_f(t, u), j & 1, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          const float f = f_share[t * 128 + ct];
-          if (__any_sync(0xffffffffu, f != 1.f)) {          // never for the first tile
-            // O must be quiescent: P V of every earlier tile of this set complete
-            ok = mbar_wait(bar_pvdone(t), (j - 1) & 1, abort_flag);
+          const float f = f_share[(t * 2 + u) * 128 + ct];
+          if (__any_sync(0xffffffffu, f != 1.f)) {          // never for the first block
+            // O must be quiescent: P V of every earlier block of this set complete
+            ok = mbar_wait(bar_pvdone(t), (b - 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -533,7 +457,7 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             tc_fence_before();
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(leader_addr(bar_corr(t)));
+          if (lane == 0) mbar_arrive_cluster(leader_addr(bar_corr(t, u)));
         }
       }
     }
@@ -542,36 +466,38 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   }
   else {
     // =========================== softmax: warps 4-7 set X, warps 8-11 set Y ===========================
-    // One thread per query row: the row's 128 scores of a key tile sit in its registers, so the
-    // maximum and the sum need no exchange with other threads.
-    reg_acquire<kRegsSoftmax>();
+    // One thread per query row: the row's 64 scores of a block sit in its registers, so the maximum
+    // and the sum need no exchange with other threads.
     const int t = warp >= 8 ? 1 : 0;
     const int q4 = warp & 3, row = q4 * 32 + lane;
-    const uint32_t s_addr = tmem + (uint32_t(q4 * 32) << 16) + t * 128;
-    for (int j = 0; j < n_tiles; ++j) {
-      row_ok = mbar_wait(bar_sfull(t), j & 1, abort_flag);
+    const uint32_t s_row = tmem + (uint32_t(q4 * 32) << 16) + t * 128;
+    for (int b = 0; b < 2 * n_tiles; ++b) {
+      const int u = b & 1;
+      row_ok = mbar_wait(bar_sfull(t, u), (b >> 1) & 1, abort_flag);
       row_ok = __all_sync(0xffffffffu, row_ok);
       if (!row_ok) break;
       tc_fence_after();
-      uint64_t sv[64];                                    // sv[i] = columns 2i, 2i + 1
-      TMEM_LD128P_WAIT(s_addr, sv);
+      const uint32_t s_addr = s_row + u * kBlk;
+      uint64_t sv[32];                                    // sv[i] = columns 2i, 2i + 1 of this block
+      TMEM_LD64P_WAIT(s_addr, sv);
       // key-validity limit: ragged last past tile, or the causal diagonal of the last tile
-      const int jj = j_lo + j;
+      const int jj = j_lo + (b >> 1);
       int lim = kBN;
       if (jj < past_tiles) lim = min(kBN, n_past - jj * kBN);
       else if (jj == all_tiles - 1) lim = row + 1;
+      lim -= u * kBlk;                                    // in this block's column numbering
       const bool masked = (jj == all_tiles - 1) || (jj == past_tiles - 1 && (n_past % kBN) != 0);   // CTA-uniform
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
       if (masked) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
+        for (int i = 0; i < 32; ++i) {
           const float a0 = 2 * i < lim ? lo2(sv[i]) : -INFINITY, a1 = 2 * i + 1 < lim ? hi2(sv[i]) : -INFINITY;
           sv[i] = pack2(a0, a1);
           mx0 = max3(mx0, a0, a1);
         }
       } else {
 #pragma unroll
-        for (int i = 0; i < 64; i += 4) {                 // four chains
+        for (int i = 0; i < 32; i += 4) {                 // four chains
           mx0 = max3(mx0, lo2(sv[i]), hi2(sv[i]));
           mx1 = max3(mx1, lo2(sv[i + 1]), hi2(sv[i + 1]));
           mx2 = max3(mx2, lo2(sv[i + 2]), hi2(sv[i + 2]));
@@ -579,22 +505,23 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
       }
       const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      // (a block of the diagonal tile can be masked entirely for a row: mx = -inf, nothing changes)
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const bool grow = m_new - m_run > kRescaleF16;      // also true for the first tile
-      // Where the maximum grew, O has to be scaled by f before P(j) V(j) is added: the correction
-      // warps do that, off this thread's path; the first tile starts O, so its factor is 1.
+      const bool grow = m_new - m_run > kRescaleF16;      // also true for the first block
+      // Where the maximum grew, O has to be scaled by f before P(b) V(b) is added: the correction
+      // warps do that, off this thread's path; the first block starts O, so its factor is 1.
       const float f = grow ? ex2(m_run - m_new) : 1.f;
-      f_share[t * 128 + row] = j > 0 ? f : 1.f;
+      f_share[(t * 2 + u) * 128 + row] = b > 0 ? f : 1.f;
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_f(t));
+      if (lane == 0) mbar_arrive(bar_f(t, u));
       if (grow) { m_run = m_new; l_run *= f; }
-      // P = exp2(x - m) in fp16, written over the first 64 columns of this row of S (all of which
-      // this thread already holds).  The row sum adds the values as rounded to fp16, the ones
-      // P V multiplies, so numerator and denominator carry the same rounding.
+      // P = exp2(x - m) in fp16, written over the first 32 columns of this row of the S buffer (all
+      // of which this thread already holds).  The row sum adds the values as rounded to fp16, the
+      // ones P V multiplies, so numerator and denominator carry the same rounding.
       const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), negm = pack2(-m_run, -m_run);
       float sa = 0.f, sb = 0.f;
 #pragma unroll
-      for (int cq = 0; cq < 4; ++cq) {
+      for (int cq = 0; cq < 2; ++cq) {
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
@@ -608,7 +535,7 @@ attention_tc4_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();                                       // one arrival per warp: 8 of both CTAs' warps of this set
-      if (lane == 0) mbar_arrive_cluster(leader_addr(bar_pfull(t)));
+      if (lane == 0) mbar_arrive_cluster(leader_addr(bar_pfull(t, u)));
     }
     // the last P V depends, through the softmax, on every Q K^T: O is final once this completes
     if (n_tiles > 0) {
@@ -732,7 +659,7 @@ int launch_attention_tc4(const actqkv_config* cfg, const Batch& b, const AttnArg
   {
     const cuuint64_t dims[3] = {cuuint64_t(kD), cuuint64_t(Hkv), cuuint64_t(U) * nt};
     const cuuint64_t str[2] = {cuuint64_t(kD) * 2, cuuint64_t(Hkv) * kD * 2};
-    const cuuint32_t box_k[3] = {64, 1, 64};                       // one channel half of 64 keys
+    const cuuint32_t box_k[3] = {64, 1, 32};                       // one channel half of 32 keys
     const cuuint32_t box_v[3] = {64, 1, cuuint32_t(kBN)};          // one channel half of 128 keys
     if (!encode(&tm_kw, a.k_win, 3, dims, str, box_k)) return ACTQKV_ERR_LAUNCH;
     if (!encode(&tm_vw, a.v_win, 3, dims, str, box_v)) return ACTQKV_ERR_LAUNCH;

@@ -29,7 +29,7 @@ inline int check_config(const actqkv_config* c, const Batch& b) {
   if (c->dtype != ACTQKV_F32 && c->dtype != ACTQKV_BF16) return ACTQKV_ERR_DTYPE;
   if (c->out_dtype != ACTQKV_F32 && c->out_dtype != ACTQKV_BF16) return ACTQKV_ERR_DTYPE;
   if (c->probe_mode != ACTQKV_PROBE_ACTIVATION && c->probe_mode != ACTQKV_PROBE_MEAN_POOL) return ACTQKV_ERR_SHAPE;
-  if (c->attention_kernel < ACTQKV_ATTN_AUTO || c->attention_kernel > ACTQKV_ATTN_PAIR) return ACTQKV_ERR_SHAPE;
+  if (c->attention_kernel < ACTQKV_ATTN_AUTO || c->attention_kernel > ACTQKV_ATTN_CLUSTER4) return ACTQKV_ERR_SHAPE;
   if (c->head_dim != 64 && c->head_dim != 128) return ACTQKV_ERR_SHAPE;
   if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_q_heads % c->n_kv_heads) return ACTQKV_ERR_SHAPE;
   if (c->n_q_heads / c->n_kv_heads > 8) return ACTQKV_ERR_SHAPE;

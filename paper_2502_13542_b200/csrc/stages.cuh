@@ -50,7 +50,7 @@ int launch_attention_tc(const actqkv_config* cfg, const Batch& b, const AttnArgs
 bool attention_tc2_supported(const actqkv_config* cfg, int n_tokens);
 int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 // Four query heads of a KV group per CTA pair, the key stream split over the two pairs of a 4-CTA
-// cluster (needs a multiple of 4 query heads per KV head).
+// cluster (needs a multiple of 4 query heads per KV head).  Not the default: see attention_tc4.cu.
 bool attention_tc4_supported(const actqkv_config* cfg, int n_tokens);
 int launch_attention_tc4(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st);
 

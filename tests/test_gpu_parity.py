@@ -36,12 +36,15 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
     orc_kw = {{"agg_mode": "agg"}.get(k, k): v[1] for k, v in variant.items()}
     cfg = B.make_config(spec, beta=beta, out_dtype=out_dtype, **lib_kw)
     cfg_b = B.make_config(spec, beta=beta, out_dtype=B.BF16, **lib_kw)
+    cfg_c4 = B.make_config(spec, beta=beta, out_dtype=B.BF16, attention_kernel=B.ATTN_CLUSTER4, **lib_kw)
+    with_c4 = also_bf16_out and spec.dtype == "bf16" and spec.group % 4 == 0 and spec.window % 128 == 0
     n_pages = cfg.n_phys_pages
     pt = wl.shuffled_page_table(spec, spec.context)
     st = B.RetrievalState(cfg, page_table=pt[None, :], keep_phi=True)
     o_run = pu.OracleRunner(spec, beta=beta, **orc_kw)
     out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=cfg.torch_out_dtype, device="cuda")
     out_b = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device="cuda")
+    out_c4 = torch.zeros_like(out_b)
     lse = torch.zeros(spec.n_q_heads, spec.window, dtype=torch.float32, device="cuda")
     stats = dict(near=0, worst_att=0.0, worst_att_mean=0.0, worst_rel=0.0, fragile=0, att_checked=0,
                  att_sampled=0, worst_att_bf16=0.0)
@@ -62,6 +65,9 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
             # tokens >= p0, which this call takes from dk / dv)
             B.retrieval_attention(cfg_b, st.batch, dq, dk, dv, spec.window, st.k_pages, st.v_pages, st.page_table,
                                   st.pos0, st.sel_idx, st.sel_count, out_b, None, st.status)
+            if with_c4:           # and on the 4-CTA-cluster kernel
+                B.retrieval_attention(cfg_c4, st.batch, dq, dk, dv, spec.window, st.k_pages, st.v_pages, st.page_table,
+                                      st.pos0, st.sel_idx, st.sel_count, out_c4, None, st.status)
         st.set_positions([p0 + spec.window])
         torch.cuda.synchronize()
         assert int(st.status.item()) == 0, f"window {t}: device status {int(st.status.item())}"
@@ -106,6 +112,8 @@ def _run_sweep(B, spec, windows_with_attention, fused, check_every=True, beta=1.
             if also_bf16_out:
                 mxb, _ = pu.assert_attention_bf16_out(pu.to_numpy(out_b), res["out"], tag + " attention, bf16 output")
                 stats["worst_att_bf16"] = max(stats["worst_att_bf16"], mxb)
+                if with_c4:
+                    pu.assert_attention_bf16_out(pu.to_numpy(out_c4), res["out"], tag + " attention, cluster kernel")
             stats["att_checked"] += 1
         # step 6: table rows of the blocks completed so far are bit-identical, pages hold the cache
         nb = o_run.complete_blocks()
@@ -300,8 +308,8 @@ def test_edge_cases_and_errors(B):
 @pytest.mark.parametrize("kernel", ["cluster4", "pair", "tc1"])
 @pytest.mark.parametrize("target", [1, 3])
 def test_tc_attention_repeatable_and_matches_general_kernel(B, target, kernel):
-    """The tensor-core attention (the 4-CTA-cluster kernel the shape selects by default, the
-    CTA-pair kernel and the single-CTA kernel) is run many times on the same state: every run must give the same bits
+    """The tensor-core attention (the CTA-pair kernel the shape selects by default, the
+    4-CTA-cluster kernel and the single-CTA kernel) is run many times on the same state: every run must give the same bits
     (no timing dependence), and agree with the general fp32 kernel.  Window 1 gives the shortest
     key-tile loops (5 to 8 tiles), window 3 longer ones."""
     import torch
@@ -328,7 +336,7 @@ def test_tc_attention_repeatable_and_matches_general_kernel(B, target, kernel):
     gen = torch.zeros_like(out)
     attend(gen, B.ATTN_GENERAL)
     torch.cuda.synchronize()
-    which = {"tc1": B.ATTN_SINGLE_CTA, "pair": B.ATTN_PAIR, "cluster4": B.ATTN_AUTO}[kernel]
+    which = {"tc1": B.ATTN_SINGLE_CTA, "pair": B.ATTN_AUTO, "cluster4": B.ATTN_CLUSTER4}[kernel]
     outs = [torch.zeros_like(out) for _ in range(8)]
     ref = None
     for rep in range(60):

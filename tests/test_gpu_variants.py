@@ -99,7 +99,8 @@ def test_prefill_step_off_the_page_boundary(B):
             assert pu.compare_selection(pu.to_numpy(st.sel_idx[0]).astype(np.int64), int(st.sel_count.item()), res,
                                         f"step {t}") == 0
             pu.assert_attention(pu.to_numpy(o), res["out"], f"unaligned p0 = {p0}, pair kernel")
-            for which, nm in ((B.ATTN_SINGLE_CTA, "single-CTA kernel"), (B.ATTN_GENERAL, "general kernel")):
+            for which, nm in ((B.ATTN_SINGLE_CTA, "single-CTA kernel"), (B.ATTN_CLUSTER4, "4-CTA-cluster kernel"),
+                              (B.ATTN_GENERAL, "general kernel")):
                 c2 = B.make_config(spec, out_dtype=B.F32, attention_kernel=which)
                 o2 = torch.full_like(o, float("nan"))
                 B.retrieval_attention(c2, st.batch, dq, dk, dv, nt, st.k_pages, st.v_pages, st.page_table, st.pos0,
