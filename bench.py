@@ -174,6 +174,15 @@ def build_states(spec, n_copies, device, sweep_times=None, flush=None):
     out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, dtype=torch.bfloat16, device=device)
     T = spec.n_windows
     evs = []
+    if sweep_times is not None:
+        # first launches of every kernel (module load, shared-memory opt-in) on a scratch state
+        warm = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :], device=device)
+        for t in range(2):
+            kw, vw = wl.gen_kv(spec, 0, t)
+            warm.step(wl.to_device(wl.gen_q(spec, 0, t)[None], spec, device), wl.to_device(kw[None], spec, device),
+                      wl.to_device(vw[None], spec, device), out, overlap_append=True)
+        torch.cuda.synchronize()
+        del warm
     for t in range(T - 1):
         q = wl.to_device(wl.gen_q(spec, 0, t)[None], spec, device)
         k, v = wl.gen_kv(spec, 0, t)
@@ -323,20 +332,39 @@ def run_ours(args):
     stage_us = {k: float(np.mean(v)) for k, v in stage_all.items()}
     assert all(int(st.status.item()) == 0 for st in states), "device status set during the bench"
 
+    # The dominant kernel alone: `att_batch` launches back to back on the rotated (cold) copies between
+    # two events, repeated; the duration of one launch is the batch time / launches.  (An event pair
+    # around a single launch also counts the idle gap before the kernel starts: stages["attention"].)
+    att_batch, att_reps = max(args.steps, 20), []
+    for _ in range(5):
+        a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for i in range(att_batch):
+            st = states[i % n_copies]
+            q_, k_, v_, o_ = inputs[i % n_copies]
+            B.retrieval_attention(cfg, st.batch, q_, k_, v_, spec.window, st.k_pages, st.v_pages, st.page_table,
+                                  st.pos0, st.sel_idx, st.sel_count, o_, None, st.status)
+        a1.record()
+        torch.cuda.synchronize()
+        att_reps.append(1e3 * a0.elapsed_time(a1) / att_batch)
+    att_us = float(np.median(att_reps))
     c_sel = int(states[0].sel_count.item())
     flops = attention_flops(spec, p0, c_sel)
-    att_tflops = flops / (stage_us["attention"] * 1e-6) / 1e12
+    att_tflops = flops / (att_us * 1e-6) / 1e12
     peak = peaks["bf16_tflops"]
     roofline = {"bound": "tensor", "kernel": "retrieval_attention", "achieved": att_tflops, "peak": peak,
                 "unit": "TFLOP/s", "frac": att_tflops / peak, "traffic": attention_traffic(),
-                "peak_source": peaks["source"] + " burst bf16 (cuBLAS)", "flops_per_launch": flops}
+                "peak_source": peaks["source"] + " burst bf16 (cuBLAS)", "flops_per_launch": flops,
+                "us_per_launch": att_us, "launches_timed": att_batch * len(att_reps),
+                "timing": f"CUDA events around {att_batch} back-to-back launches on rotated cold copies, median of {len(att_reps)} batches",
+                "us_single_launch_between_events": float(np.median(stage_all["attention"]))}
     sb = stage_bytes(spec, p0)
     stages = {k: {"us": v, "median_us": float(np.median(stage_all[k])), "min_us": float(np.min(stage_all[k]))}
               for k, v in stage_us.items()}
     stages["bias_probe"]["GBps"] = sb["bias_probe"] / stage_us["bias_probe"] / 1e3
     stages["score_select"]["GBps"] = (sb["score"] + sb["select"]) / stage_us["score_select"] / 1e3
     stages["append"]["GBps"] = sb["append"] / stage_us["append"] / 1e3
-    stages["attention"]["TFLOPs"] = att_tflops
+    stages["attention"]["TFLOPs"] = flops / (stage_us["attention"] * 1e-6) / 1e12
 
     # end to end through the public API with host buffers (pinned), copies inside the timed region
     q, k, v, out = inputs[0]

@@ -130,6 +130,12 @@ typedef struct actqkv_config {
   int32_t out_dtype;     /* element type of the attention output: ACTQKV_F32 | ACTQKV_BF16 */
   int32_t probe_mode;    /* ACTQKV_PROBE_*: token weights of the probe-query                 */
   int32_t attention_kernel; /* ACTQKV_ATTN_*: 0 = pick by shape                              */
+  /* Test hooks of the failure-detection path (leave both 0).  With test_wait_limit > 0 the decode
+   * attention kernel gives its device-side waits that many polls instead of the normal 2^24 and
+   * never issues the K copy of tile test_drop_k_tile of each CTA, so that the wait for that tile runs
+   * out: the kernel must set ACTQKV_DEV_TIMEOUT, return, and leave the context usable. */
+  int32_t test_wait_limit;
+  int32_t test_drop_k_tile;
 } actqkv_config;
 
 typedef struct actqkv_batch {

@@ -40,7 +40,8 @@ class Config(C.Structure):
         "n_init", "n_local_prev", "k_blocks", "cap_blocks", "dtype", "stats_mode", "repr_mode",
         "agg_mode", "thetabar_mode", "n_cap", "max_pages", "n_phys_pages")] + [
         ("beta", C.c_float), ("sm_scale", C.c_float), ("var_eps", C.c_float), ("out_dtype", C.c_int32),
-        ("probe_mode", C.c_int32), ("attention_kernel", C.c_int32)]
+        ("probe_mode", C.c_int32), ("attention_kernel", C.c_int32), ("test_wait_limit", C.c_int32),
+        ("test_drop_k_tile", C.c_int32)]
 
     @property
     def torch_dtype(self):

@@ -44,6 +44,8 @@ static_assert(kSmemNeeded <= kSmemBytes, "shared memory budget");
 
 
 struct DecodeParams {
+  uint32_t spin_limit; // iterations a device-side wait may take (kSpinLimit; shorter only under test)
+  int drop_k_tile;     // test hook: the K copy of this tile of every CTA is not issued (-1: none)
   int n_splits;        // CTAs per (unit, KV head)
   float* part_o;       // [U][n_tokens][Hq][n_splits][D] normalised partial outputs (n_splits > 1)
   float* part_lse;     // [U][n_tokens][Hq][n_splits] base-2 log-sum-exp of each split (-inf: empty)
@@ -180,14 +182,16 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       const int s = j % kRing, it = j / kRing;
       if ((j & 3) == 0) page_cur = page_next;
       const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + slot);
-      if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
+      if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag, dp.spin_limit);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const uint32_t full = is_v ? bar_vfull(s) : bar_kfull(s);
       const uint32_t sbase = ring + s * kTileBytes;
-      if (lane == 0) mbar_expect_tx(full, kTileBytes);
+      const bool dropped = !is_v && j == dp.drop_k_tile;   // test hook: this copy is never made, so the wait for it runs out
+      if (lane == 0 && !dropped) mbar_expect_tx(full, kTileBytes);
       __syncwarp();
-      if (j_lo + j < past_tiles) {
+      if (dropped) {
+      } else if (j_lo + j < past_tiles) {
         if (lane < 16) tma_load_4d(sbase + half * kSubTileBytes + slot * 2048u, tm_pages, full, half * 64, 0, g, page);
       } else if (lane < 2) {
         tma_load_3d(sbase + lane * kSubTileBytes, tm_win, full, lane * 64, g, unit * nt);
@@ -198,10 +202,11 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     // drain: every issued copy must have landed before the CTA may exit on the abort path
     if (!ok) {
       for (int j = max(0, issued - kRing); j < issued; ++j) {
+        if (!is_v && j == dp.drop_k_tile) continue;
         const uint32_t full = is_v ? bar_vfull(j % kRing) : bar_kfull(j % kRing);
-        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(full, (j / kRing) & 1); ++i) {}
+        for (uint32_t i = 0; i < dp.spin_limit && !mbar_try_wait(full, (j / kRing) & 1); ++i) {}
       }
-      if (!is_v) for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(bar_q, 0); ++i) {}
+      if (!is_v) for (uint32_t i = 0; i < dp.spin_limit && !mbar_try_wait(bar_q, 0); ++i) {}
     }
   } else if (warp == 1) {
     // =========================== MMA issuer ===========================
@@ -209,10 +214,10 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       constexpr uint32_t idesc_qk = make_idesc(false, kBM, kBN);
       constexpr uint32_t idesc_pv = make_idesc(true, kBM, kBN);
       const uint32_t tmem_o = tmem + kSBuf * 128;
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      bool ok = mbar_wait(bar_q, 0, abort_flag, dp.spin_limit);
       auto issue_qk = [&](int j) {
         const int s = j % kRing;
-        ok = ok && mbar_wait(bar_kfull(s), (j / kRing) & 1, abort_flag);
+        ok = ok && mbar_wait(bar_kfull(s), (j / kRing) & 1, abort_flag, dp.spin_limit);
         if (!ok) return;
         tc_fence_after();
         const uint32_t kbase = k_ring + s * kTileBytes;
@@ -228,8 +233,8 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       };
       auto issue_pv = [&](int i) {
         const int s = i % kRing, b = i % kSBuf;
-        ok = ok && mbar_wait(bar_vfull(s), (i / kRing) & 1, abort_flag);
-        ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag);
+        ok = ok && mbar_wait(bar_vfull(s), (i / kRing) & 1, abort_flag, dp.spin_limit);
+        ok = ok && mbar_wait(bar_pfull(b), (i / kSBuf) & 1, abort_flag, dp.spin_limit);
         if (!ok) return;
         tc_fence_after();
         const uint32_t vbase = v_ring + s * kTileBytes;
@@ -252,7 +257,10 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         if (i + 2 < n_tiles) issue_qk(i + 2);
         issue_pv(i);
       }
-      if (ok) tc_commit(bar_done);
+      tc_commit(bar_done);
+      // when a wait gave up nobody else waits for this barrier: the issuer itself sees the products
+      // it has issued through, so that TMEM is not freed under them
+      if (!ok) for (uint32_t i = 0; i < dp.spin_limit && !mbar_try_wait(bar_done, 0); ++i) {}
     }
     __syncwarp();
   } else if (warp >= 4) {
@@ -271,13 +279,13 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     if (!warp_used) {
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int sb = j % kSBuf;
-        ok = mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
+        ok = mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag, dp.spin_limit);
         mbar_arrive(bar_pfull(sb));
       }
     }
     for (int j = 0; warp_used && j < n_tiles; ++j) {
       const int sb = j % kSBuf;
-      ok = ok && mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
+      ok = ok && mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag, dp.spin_limit);
       tc_fence_after();
       const uint32_t s_addr = tmem + lane_addr + sb * 128 + b * 64;
       uint64_t sv[32];
@@ -323,7 +331,7 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         // O must be quiescent: P V of every earlier tile complete (tile j's is not issued before
         // this thread publishes P(j)).  One barrier per tile in a ring of 4, so the parity of the
         // awaited phase cannot be confused with a later one.
-        ok = mbar_wait(bar_pvdone((j - 1) % kPvRing), ((j - 1) / kPvRing) & 1, abort_flag);
+        ok = mbar_wait(bar_pvdone((j - 1) % kPvRing), ((j - 1) / kPvRing) & 1, abort_flag, dp.spin_limit);
         tc_fence_after();
         const float f = grow ? ex2(m_used - m_new) : 1.f;
         if (grow) { m_used = m_new; l *= f; }
@@ -363,7 +371,7 @@ attention_decode_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       mbar_arrive(bar_pfull(sb));
     }
     // ---- epilogue: the row sum over both column halves, then this thread's 64 channels of O / l
-    ok = ok && warp_used && mbar_wait(bar_done, 0, abort_flag);
+    ok = ok && warp_used && mbar_wait(bar_done, 0, abort_flag, dp.spin_limit);
     float* xrow = xchg + (n_tiles & 1) * 256 + row;
     if (warp_used) {
       xrow[b * 128] = l;
@@ -531,6 +539,8 @@ int launch_attention_decode(const actqkv_config* cfg, const Batch& b, const Attn
   const float scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.f / sqrtf(float(kD));
   p.scale_log2 = scale * 1.4426950408889634f;
   DecodeParams dp;
+  dp.spin_limit = cfg->test_wait_limit > 0 ? uint32_t(cfg->test_wait_limit) : kSpinLimit;
+  dp.drop_k_tile = cfg->test_wait_limit > 0 ? cfg->test_drop_k_tile : -1;
   dp.n_splits = std::max(1, n_splits);
   const size_t rows = size_t(U) * nt * Hq;
   dp.part_o = static_cast<float*>(workspace);

@@ -366,89 +366,104 @@ bool encode_q(CUtensorMap* tm, const BiasProbeParams& p, int units, int box_rows
 
 // ---------------------------------------------------------------------------------------------
 // Batched calls (many (unit, head) items, e.g. all layers of a model in one launch): a persistent
-// kernel, one CTA per SM, no clusters.  A CTA takes whole items: the [n_tokens x D] tile of one
-// head arrives as up to kMaxChunks row chunks, one tiled TMA load and one barrier each; the column
-// sums of pass 1 are taken chunk by chunk while later chunks are still in flight; after the
-// statistics are merged a single second pass computes phi, the indicator a_j = ||phi_j||_1 and
-// sum_j a_j q_j together (the row is still in registers when its a_j is known), and hands every
-// chunk it has finished to the load of the CTA's NEXT item, so the loads never stop.  (A variant
-// in which every thread copied its own vectors with cp.async, without barriers, was slower: the
-// stage is bound by its instruction count, and the copies add to it.)  The KV-head probes (mean
-// over the G heads of a group, Eq. 9) are taken from the stored per-head probes by a small second
-// kernel.
-#ifndef MAX_CHUNKS
-#define MAX_CHUNKS 2
-#endif
-constexpr int kMaxChunks = MAX_CHUNKS;
-#ifndef STREAM_THREADS
-#define STREAM_THREADS 512
-#endif
-constexpr int kStreamThreads = STREAM_THREADS;
+// kernel without clusters.  A CTA is small enough for TWO to share an SM -- eight consumer warps and
+// one producer warp, 16 KiB chunks in a ring of four slots -- so that the reductions and barrier
+// waits of one CTA's item are filled with the row passes of the other's.  An item is not kept in
+// shared memory: the producer brings its chunks once for pass 1 (column sums -> statistics, Eq. 8)
+// and once more for pass 2 (phi, a_j = ||phi_j||_1 and sum_j a_j q_j, Eq. 7 and 9); the second read
+// is served by L2 (two items per SM are 256 KiB in flight out of 126 MB), so HBM still sees every
+// query once and n_tokens is not limited by the shared memory.  Slots are handed over with
+// full / empty mbarriers (the producer never takes part in a CTA barrier); every wait is bounded.
+// The kernel is bound by its instruction pipes, not by memory or latency: a form that kept one whole
+// item per SM in shared memory (16 warps, phases in series) took the same 57 us for 32 layers,
+// three CTAs per SM are slower, and the packed fp32 and integer pipes both run at one warp
+// instruction per two cycles, which the unpacking of bf16 pairs and the 24 packed operations per
+// 16-byte vector fill.
+constexpr int kRingThreads = 256;           // consumer threads; warp 8 is the producer
+constexpr int kRingSlots = 4;
+constexpr int kRingCtasPerSm = 2;           // three per SM (72 registers, 3 slots) measured slower: 87 us against 62.5
+constexpr int kRingRowsPerThread = 4;       // rows of a chunk per consumer thread
+
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kRingThreads) : "memory"); }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kStreamThreads, 1)
-bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams p, int n_items, int chunk_rows, int n_chunks) {
+__global__ void __launch_bounds__(kRingThreads + 32, kRingCtasPerSm)
+bias_probe_ring_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams p, int n_items, int n_chunks) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int VN = Vec16<T>::N;
   constexpr int VPR = D / VN;
-  constexpr int RL = kStreamThreads / VPR;
-  constexpr int NP = kStreamThreads / D;
-  constexpr int NW = kStreamThreads / 32;     // warps
-  constexpr int PER = NW / NP;                // warps per second-level slice
+  constexpr int RL = kRingThreads / VPR;            // row lanes
+  constexpr int NW = kRingThreads / 32;             // consumer warps
   constexpr int N2 = Pairs<T>::N2;
+  constexpr int kChunkRows = RL * kRingRowsPerThread;
+  constexpr uint32_t kChunkBytes = uint32_t(kChunkRows) * D * sizeof(T);      // 16 KiB for every supported shape
   const int W = p.n_tokens;
-  const int rows_alloc = chunk_rows * n_chunks;
-  T* tile = reinterpret_cast<T*>(smem_raw);
-  float* partial = reinterpret_cast<float*>(smem_raw + ((size_t(rows_alloc) * D * sizeof(T) + 127) & ~size_t(127)));   // [2][NW][D]
-  float* level2 = partial + 2 * NW * D;       // [2][NP][D]
-  float* sum_a = level2 + 2 * NP * D;         // [D] first result of a column reduction
+  T* ring = reinterpret_cast<T*>(smem_raw);                                   // [kRingSlots][kChunkRows][D]
+  float* partial = reinterpret_cast<float*>(smem_raw + kRingSlots * kChunkBytes);   // [2][NW][D]
+  float* sum_a = partial + 2 * NW * D;        // [D] first result of a column reduction
   float* sum_b = sum_a + D;                   // [D] second result
   float* mean_s = sum_b + D;                  // [D]
   float* ivar_s = mean_s + D;                 // [D]
   float* qsum_s = ivar_s + D;                 // [D] sum_j q_j of the item
-  float* red_s = qsum_s + D;                  // [32]
+  float* shift_s = qsum_s + D;                // [D] row 0 of the item (the shift of pass 1)
+  float* red_s = shift_s + D;                 // [32]
   float* a_s = red_s + 32;                    // [W]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(a_s + ((W + 3) & ~3));   // [kMaxChunks]
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(a_s + ((W + 3) & ~3));     // [kRingSlots]
+  uint64_t* bar_empty = bar_full + kRingSlots;                                // [kRingSlots]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int cv = tid % VPR, rsub = tid / VPR;
-  const int passes_per_chunk = chunk_rows / RL;
-  const size_t row_stride = size_t(p.n_q_heads) * D;
-  constexpr uint32_t kRowBytes = D * sizeof(T);
   const bool running = p.do_bias && p.stats_mode == ACTQKV_STATS_CUMULATIVE;
+  const int n_pass = p.do_bias ? 2 : 1;
 
   grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
   grid_launch_dependents();
   if (tid == 0) {
-    for (int c = 0; c < n_chunks; ++c) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bars + c)));
+    for (int s = 0; s < kRingSlots; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bar_full + s)));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar_empty + s)), "n"(NW));
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();
+  __syncthreads();                   // the only barrier the producer warp takes part in
 
-  // Rows [c * chunk_rows, (c + 1) * chunk_rows) of an item -> shared memory (rows past n_tokens
-  // belong to the next unit or are zero fill; they are never read).  Every thread of the CTA has
-  // finished with the chunk's previous contents when this is called (a CTA barrier precedes it).
-  auto issue_chunk = [&](int item, int c) {
-    if (tid == 0) {
-      const int unit = item / p.n_q_heads, h = item - unit * p.n_q_heads;
-      const uint32_t bar = smem_addr(bars + c);
-      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(uint32_t(chunk_rows) * kRowBytes) : "memory");
-      tc::tma_load_3d(smem_addr(tile + size_t(c) * chunk_rows * D), &tm_q, bar, 0, h, unit * W + c * chunk_rows);
-    }
-  };
-  auto wait_chunk = [&](int c, uint32_t parity) {
-    const uint32_t bar = smem_addr(bars + c);
-    bool landed = false;
-    for (uint32_t i = 0; i < kSpinLimit && !landed; ++i) {
+  auto wait_bar = [&](uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_addr(bar);
+    bool done = false;
+    for (uint32_t i = 0; i < kSpinLimit && !done; ++i) {
       uint32_t ok;
       asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                   : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-      landed = ok != 0;
+                   : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+      done = ok != 0;
     }
-    if (!landed && tid == 0) set_status(p.status, ACTQKV_DEV_TIMEOUT);     // goes on with whatever arrived
+    if (!done && lane == 0) set_status(p.status, ACTQKV_DEV_TIMEOUT);     // goes on with whatever arrived
   };
-  // dst0 / dst1 [D] = sums over the row lanes of a0 / a1, in a fixed order: the rows of a warp by
-  // shuffles, then the warps in two levels through shared memory (16-byte stores, no bank conflicts)
+
+  if (warp == NW) {
+    // =========================== producer: one thread walks the load sequence ===========================
+    // item by item: its chunks for pass 1, then the same chunks for pass 2.  Rows past n_tokens belong
+    // to the next unit or are zero fill; they are never read.
+    if (lane == 0) {
+      uint32_t seq = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int unit = item / p.n_q_heads, h = item - unit * p.n_q_heads;
+        for (int pass = 0; pass < n_pass; ++pass)
+          for (int c = 0; c < n_chunks; ++c, ++seq) {
+            const uint32_t slot = seq % kRingSlots, round = seq / kRingSlots;
+            if (round > 0) wait_bar(bar_empty + slot, (round - 1) & 1);
+            const uint32_t bar = smem_addr(bar_full + slot);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kChunkBytes) : "memory");
+            tc::tma_load_3d(smem_addr(ring + size_t(slot) * kChunkRows * D), &tm_q, bar, 0, h, unit * W + c * kChunkRows);
+          }
+      }
+    }
+    return;
+  }
+
+  // =========================== consumers ===========================
+  const int cv = tid % VPR, rsub = tid / VPR;
+  const size_t row_stride = size_t(p.n_q_heads) * D;
+  // dst0 / dst1 [D] = sums over the row lanes of a0 / a1 in a fixed order: the rows of a warp by
+  // shuffles, then the eight warps through shared memory
   auto column_reduce2 = [&](float (&a0)[VN], float (&a1)[VN], float* dst0, float* dst1) {
 #pragma unroll
     for (int o = VPR; o < 32; o <<= 1) {
@@ -458,7 +473,7 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
         a1[e] += __shfl_xor_sync(0xffffffffu, a1[e], o);
       }
     }
-    __syncthreads();
+    consumer_barrier();                              // earlier readers of `partial` are done
     if (lane < VPR) {
 #pragma unroll
       for (int e = 0; e < VN; e += 4) {
@@ -466,38 +481,22 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
         *reinterpret_cast<float4*>(partial + NW * D + warp * D + cv * VN + e) = make_float4(a1[e], a1[e + 1], a1[e + 2], a1[e + 3]);
       }
     }
-    __syncthreads();
-    {
-      const int ch = tid % D, part = tid / D;
-      float t0 = 0.f, t1 = 0.f;
+    consumer_barrier();
+    for (int ch = tid; ch < 2 * D; ch += kRingThreads) {
+      const float* src = partial + (ch >= D ? NW * D : 0) + (ch % D);
+      float t = 0.f;
 #pragma unroll
-      for (int q = 0; q < PER; ++q) {
-        t0 += partial[(part * PER + q) * D + ch];
-        t1 += partial[NW * D + (part * PER + q) * D + ch];
-      }
-      level2[part * D + ch] = t0;
-      level2[NP * D + part * D + ch] = t1;
+      for (int w = 0; w < NW; ++w) t += src[w * D];
+      (ch >= D ? dst1 : dst0)[ch % D] = t;
     }
-    __syncthreads();
-    if (tid < D) {
-      float t0 = 0.f, t1 = 0.f;
-#pragma unroll
-      for (int q = 0; q < NP; ++q) { t0 += level2[q * D + tid]; t1 += level2[NP * D + q * D + tid]; }
-      dst0[tid] = t0;
-      dst1[tid] = t1;
-    }
-    __syncthreads();
+    consumer_barrier();
   };
 
-  if (int(blockIdx.x) < n_items)
-    for (int c = 0; c < n_chunks; ++c) issue_chunk(blockIdx.x, c);
-
-  uint32_t parity = 0;
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x, parity ^= 1) {
+  uint32_t seq = 0;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
     const int unit = item / p.n_q_heads, h = item - unit * p.n_q_heads;
     const size_t hd = (size_t(unit) * p.n_q_heads + h) * D;
     const size_t uh = size_t(unit) * p.n_q_heads + h;
-    const int next = item + gridDim.x;
     float run_mean = 0.f, run_m2 = 0.f;
     int64_t run_count = 0;
     if (running && tid < D) {
@@ -511,22 +510,34 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
       uint64_t shift2[N2], s1p[N2], s2p[N2];
 #pragma unroll
       for (int e = 0; e < N2; ++e) { s1p[e] = 0; s2p[e] = 0; shift2[e] = 0; }
-      for (int c = 0; c < n_chunks; ++c) {
-        wait_chunk(c, parity);
-        if (c == 0) Pairs<T>::get(*reinterpret_cast<const uint4*>(tile + cv * VN), shift2);
-        const T* src = tile + size_t(c * chunk_rows + rsub) * D + cv * VN;
-        const int n_here = min(passes_per_chunk, (W - c * chunk_rows - rsub + RL - 1) / RL);   // rows of this lane in the chunk
-#pragma unroll 2
-        for (int k = 0; k < n_here; ++k) {
-          uint64_t x[N2];
-          Pairs<T>::get(*reinterpret_cast<const uint4*>(src + size_t(k) * RL * D), x);
+      for (int c = 0; c < n_chunks; ++c, ++seq) {
+        const uint32_t slot = seq % kRingSlots;
+        wait_bar(bar_full + slot, (seq / kRingSlots) & 1);
+        const T* chunk = ring + size_t(slot) * kChunkRows * D;
+        if (c == 0) {
+          Pairs<T>::get(*reinterpret_cast<const uint4*>(chunk + cv * VN), shift2);
+          for (int ch = tid; ch < D; ch += kRingThreads) shift_s[ch] = to_f32(chunk[ch]);
+        }
+        const T* src = chunk + size_t(rsub) * D + cv * VN;
+        const int r0 = c * kChunkRows + rsub;
+        uint4 raw[kRingRowsPerThread];                 // all four loads in flight before the first use
 #pragma unroll
-          for (int e = 0; e < N2; ++e) {
-            const uint64_t d = tc::sub2(x[e], shift2[e]);
-            s1p[e] = tc::add2(s1p[e], x[e]);
-            s2p[e] = tc::fma2(d, d, s2p[e]);
+        for (int k = 0; k < kRingRowsPerThread; ++k) raw[k] = *reinterpret_cast<const uint4*>(src + size_t(k) * RL * D);
+#pragma unroll
+        for (int k = 0; k < kRingRowsPerThread; ++k) {
+          if (r0 + k * RL < W) {
+            uint64_t x[N2];
+            Pairs<T>::get(raw[k], x);
+#pragma unroll
+            for (int e = 0; e < N2; ++e) {
+              const uint64_t d = tc::sub2(x[e], shift2[e]);
+              s1p[e] = tc::add2(s1p[e], x[e]);
+              s2p[e] = tc::fma2(d, d, s2p[e]);
+            }
           }
         }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar_empty + slot)) : "memory");
       }
       float s1[VN], s2[VN];
 #pragma unroll
@@ -538,7 +549,7 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
       // ---- statistics of the window, merged into the running ones (Eq. 8)
       if (tid < D) {
         double n = double(W);
-        const double sh0 = double(to_f32(tile[tid]));
+        const double sh0 = double(shift_s[tid]);
         const double sq = double(sum_a[tid]), b2 = double(sum_b[tid]);
         const double a = sq - n * sh0;             // sum (q - shift)
         double mean = sq / n, m2 = fmax(b2 - a * a / n, 0.0);
@@ -558,9 +569,9 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
         ivar_s[tid] = float(1.0 / fmax(var, double(p.var_eps)));
       }
     } else {
-      for (int r = tid; r < W; r += kStreamThreads) a_s[r] = p.phi_l1[uh * W + r];
+      for (int r = tid; r < W; r += kRingThreads) a_s[r] = p.phi_l1[uh * W + r];
     }
-    __syncthreads();
+    consumer_barrier();
     // ---- pass 2: phi, a_j = ||phi_j||_1 (Eq. 7) and this head's sum_j a_j q_j (and sum_j q_j when
     // pass 1 did not run), on packed pairs of channels
     uint64_t accp[N2], qsp[N2], mc2[N2], iv2[N2];
@@ -571,97 +582,103 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
       iv2[e] = p.do_bias ? tc::pack2(ivar_s[cv * VN + 2 * e], ivar_s[cv * VN + 2 * e + 1]) : 0;
     }
     float a_tot = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
-      if (!p.do_bias) wait_chunk(c, parity);
-      const int r_base = c * chunk_rows + rsub;
-      const T* src = tile + size_t(r_base) * D + cv * VN;
-      // the row lanes of a warp run the same number of passes (a warp holds whole rows; W < r only
-      // switches the row off), so the shuffles below are convergent
-      int k_done = 0;
-      if (p.do_bias && p.do_probe && !p.phi_full && VPR >= 4) {
-        // four rows at a time: their four sums over the VPR lanes of a row are reduced together
-        // (halves swap row pairs, quarters swap rows: 3 + log2(VPR / 4) shuffles instead of
-        // 4 log2(VPR)) and handed back to every lane of the row by four more
-        for (; k_done + 4 <= passes_per_chunk; k_done += 4) {
-          uint64_t x[4][N2];
-          float part[4];
+    const bool four_rows = p.do_bias && p.do_probe && !p.phi_full && VPR >= 4;
+    // ||phi_j||_1 is summed as sum_c q (q iv - 2 mean iv) + sum_c mean^2 iv: two packed operations per
+    // pair of channels instead of three, on both paths alike (so every form of the call gives the same
+    // bits); the full phi, when asked for, is written as (q - mean)^2 iv.
+    uint64_t nb2[N2];
+    float phi_const = 0.f;                            // this thread's channels of sum_c mean^2 iv
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const bool live = r_base + (k_done + j) * RL < W;
-            Pairs<T>::get(live ? *reinterpret_cast<const uint4*>(src + size_t(k_done + j) * RL * D) : make_uint4(0, 0, 0, 0), x[j]);
-            uint64_t part2 = 0;
+    for (int e = 0; e < N2; ++e) {
+      const uint64_t mi = tc::mul2(mc2[e], iv2[e]);
+      nb2[e] = tc::mul2(mi, tc::pack2(-2.f, -2.f));
+      const uint64_t mm = tc::mul2(mi, mc2[e]);
+      phi_const += tc::lo2(mm) + tc::hi2(mm);
+    }
+    for (int c = 0; c < n_chunks; ++c, ++seq) {
+      const uint32_t slot = seq % kRingSlots;
+      wait_bar(bar_full + slot, (seq / kRingSlots) & 1);
+      const T* src = ring + size_t(slot) * kChunkRows * D + size_t(rsub) * D + cv * VN;
+      const int r_base = c * kChunkRows + rsub;
+      // the row lanes of a warp run the same passes (a warp holds whole rows; r >= W only switches
+      // the row off), so the shuffles below are convergent
+      if (four_rows) {
+        // the thread's four rows of the chunk at once: their four sums over the VPR lanes of a row are
+        // reduced together (halves swap row pairs, quarters swap rows: 3 + log2(VPR / 4) shuffles
+        // instead of 4 log2(VPR)) and handed back to every lane of the row by four more
+        uint64_t x[4][N2];
+        float part[4];
 #pragma unroll
-            for (int e = 0; e < N2; ++e) {
-              const uint64_t d = tc::sub2(x[j][e], mc2[e]);
-              part2 = tc::fma2(tc::mul2(d, d), iv2[e], part2);
-            }
-            part[j] = live ? tc::lo2(part2) + tc::hi2(part2) : 0.f;
-          }
-          constexpr int H1 = VPR / 2, H2 = VPR / 4;
-          const bool up1 = lane & H1, up2 = lane & H2;
-          const float t0 = __shfl_xor_sync(0xffffffffu, up1 ? part[0] : part[2], H1);
-          const float t1 = __shfl_xor_sync(0xffffffffu, up1 ? part[1] : part[3], H1);
-          const float k0 = (up1 ? part[2] : part[0]) + t0, k1 = (up1 ? part[3] : part[1]) + t1;
-          float kv = (up2 ? k1 : k0) + __shfl_xor_sync(0xffffffffu, up2 ? k0 : k1, H2);
-#pragma unroll
-          for (int o = H2 >> 1; o > 0; o >>= 1) kv += __shfl_xor_sync(0xffffffffu, kv, o);
-          const int row_lane0 = lane & ~(VPR - 1);           // first lane of this row's lane group
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float a = __shfl_sync(0xffffffffu, kv, row_lane0 + (j >> 1) * H1 + (j & 1) * H2);
-            const int r = r_base + (k_done + j) * RL;
-            if (r < W && cv == 0) a_s[r] = a;
-            if (cv == 0) a_tot += a;
-            const uint64_t a2 = tc::pack2(a, a);
-#pragma unroll
-            for (int e = 0; e < N2; ++e) accp[e] = tc::fma2(a2, x[j][e], accp[e]);
-          }
-        }
-      }
-#pragma unroll 2
-      for (int k = k_done; k < passes_per_chunk; ++k) {
-        const int r = r_base + k * RL;
-        const bool live = r < W;
-        uint64_t x[N2];
-        Pairs<T>::get(live ? *reinterpret_cast<const uint4*>(src + size_t(k) * RL * D) : make_uint4(0, 0, 0, 0), x);
-        float a;
-        if (p.do_bias) {
+        for (int j = 0; j < 4; ++j) {
+          const bool live = r_base + j * RL < W;
+          Pairs<T>::get(live ? *reinterpret_cast<const uint4*>(src + size_t(j) * RL * D) : make_uint4(0, 0, 0, 0), x[j]);
           uint64_t part2 = 0;
-          if (p.phi_full && live) {
-            float* dst = p.phi_full + (size_t(unit) * W + r) * row_stride + size_t(h) * D + cv * VN;
 #pragma unroll
-            for (int e = 0; e < N2; ++e) {
-              const uint64_t d = tc::sub2(x[e], mc2[e]);
-              const uint64_t ph = tc::mul2(tc::mul2(d, d), iv2[e]);
-              *reinterpret_cast<float2*>(dst + 2 * e) = make_float2(tc::lo2(ph), tc::hi2(ph));
-            }
-          }
-#pragma unroll
-          for (int e = 0; e < N2; ++e) {
-            const uint64_t d = tc::sub2(x[e], mc2[e]);
-            part2 = tc::fma2(tc::mul2(d, d), iv2[e], part2);
-          }
-          float part = live ? tc::lo2(part2) + tc::hi2(part2) : 0.f;
-#pragma unroll
-          for (int o = VPR >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-          a = part;                                // every lane of the row holds the same sum
-          if (live && cv == 0) a_s[r] = a;
-        } else {
-          a = live ? a_s[r] : 0.f;
+          for (int e = 0; e < N2; ++e) part2 = tc::fma2(x[j][e], tc::fma2(x[j][e], iv2[e], nb2[e]), part2);
+          part[j] = live ? fmaxf(tc::lo2(part2) + tc::hi2(part2) + phi_const, 0.f) : 0.f;
         }
-        if (cv == 0) a_tot += a;
-        if (p.do_probe) {
+        constexpr int H1 = VPR / 2, H2 = VPR / 4;
+        const bool up1 = lane & H1, up2 = lane & H2;
+        const float t0 = __shfl_xor_sync(0xffffffffu, up1 ? part[0] : part[2], H1);
+        const float t1 = __shfl_xor_sync(0xffffffffu, up1 ? part[1] : part[3], H1);
+        const float k0 = (up1 ? part[2] : part[0]) + t0, k1 = (up1 ? part[3] : part[1]) + t1;
+        float kv = (up2 ? k1 : k0) + __shfl_xor_sync(0xffffffffu, up2 ? k0 : k1, H2);
+#pragma unroll
+        for (int o = H2 >> 1; o > 0; o >>= 1) kv += __shfl_xor_sync(0xffffffffu, kv, o);
+        const int row_lane0 = lane & ~(VPR - 1);           // first lane of this row's lane group
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float a = __shfl_sync(0xffffffffu, kv, row_lane0 + (j >> 1) * H1 + (j & 1) * H2);
+          const int r = r_base + j * RL;
+          if (r < W && cv == 0) a_s[r] = a;
+          if (cv == 0) a_tot += a;
           const uint64_t a2 = tc::pack2(a, a);
 #pragma unroll
-          for (int e = 0; e < N2; ++e) accp[e] = tc::fma2(a2, x[e], accp[e]);
-          if (!p.do_bias) {
+          for (int e = 0; e < N2; ++e) accp[e] = tc::fma2(a2, x[j][e], accp[e]);
+        }
+      } else {
+#pragma unroll 2
+        for (int k = 0; k < kRingRowsPerThread; ++k) {
+          const int r = r_base + k * RL;
+          const bool live = r < W;
+          uint64_t x[N2];
+          Pairs<T>::get(live ? *reinterpret_cast<const uint4*>(src + size_t(k) * RL * D) : make_uint4(0, 0, 0, 0), x);
+          float a;
+          if (p.do_bias) {
+            uint64_t part2 = 0;
+            if (p.phi_full && live) {
+              float* dst = p.phi_full + (size_t(unit) * W + r) * row_stride + size_t(h) * D + cv * VN;
 #pragma unroll
-            for (int e = 0; e < N2; ++e) qsp[e] = tc::add2(qsp[e], x[e]);
+              for (int e = 0; e < N2; ++e) {
+                const uint64_t d = tc::sub2(x[e], mc2[e]);
+                const uint64_t ph = tc::mul2(tc::mul2(d, d), iv2[e]);
+                *reinterpret_cast<float2*>(dst + 2 * e) = make_float2(tc::lo2(ph), tc::hi2(ph));
+              }
+            }
+#pragma unroll
+            for (int e = 0; e < N2; ++e) part2 = tc::fma2(x[e], tc::fma2(x[e], iv2[e], nb2[e]), part2);   // as on the four-row path
+            float part = live ? fmaxf(tc::lo2(part2) + tc::hi2(part2) + phi_const, 0.f) : 0.f;
+#pragma unroll
+            for (int o = VPR >> 1; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+            a = part;                                // every lane of the row holds the same sum
+            if (live && cv == 0) a_s[r] = a;
+          } else {
+            a = live ? a_s[r] : 0.f;
+          }
+          if (cv == 0) a_tot += a;
+          if (p.do_probe) {
+            const uint64_t a2 = tc::pack2(a, a);
+#pragma unroll
+            for (int e = 0; e < N2; ++e) accp[e] = tc::fma2(a2, x[e], accp[e]);
+            if (!p.do_bias) {
+#pragma unroll
+              for (int e = 0; e < N2; ++e) qsp[e] = tc::add2(qsp[e], x[e]);
+            }
           }
         }
       }
-      __syncthreads();                             // every thread is done with chunk c (and a_s has its rows)
-      if (next < n_items) issue_chunk(next, c);
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar_empty + slot)) : "memory");
     }
     float acc[VN], qs[VN];
 #pragma unroll
@@ -669,21 +686,24 @@ bias_probe_stream_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbePara
       acc[2 * e] = tc::lo2(accp[e]); acc[2 * e + 1] = tc::hi2(accp[e]);
       qs[2 * e] = tc::lo2(qsp[e]); qs[2 * e + 1] = tc::hi2(qsp[e]);
     }
-    if (p.do_bias && p.phi_l1)
-      for (int r = tid; r < W; r += kStreamThreads) p.phi_l1[uh * W + r] = a_s[r];
     if (p.do_probe) {
       // ---- Eq. 9 for this head
       a_tot = warp_sum(a_tot);
       if (lane == 0) red_s[warp] = a_tot;
-      column_reduce2(acc, qs, sum_a, sum_b);
+      column_reduce2(acc, qs, sum_a, sum_b);         // its barriers also publish a_s and red_s
       if (tid < D) {
         float t = 0.f;
-        for (int i = 0; i < kStreamThreads / 32; ++i) t += red_s[i];
+#pragma unroll
+        for (int i = 0; i < NW; ++i) t += red_s[i];
         const float qsum = p.do_bias ? qsum_s[tid] : sum_b[tid];
         p.probe_qh[hd + tid] = (t > 0.f && !p.mean_pool) ? sum_a[tid] / t : qsum / float(W);   // all-zero bias: uniform weights
       }
+    } else {
+      consumer_barrier();                            // a_s is complete
     }
-    __syncthreads();
+    if (p.do_bias && p.phi_l1)
+      for (int r = tid; r < W; r += kRingThreads) p.phi_l1[uh * W + r] = a_s[r];
+    consumer_barrier();                              // everything of this item has been read
   }
 }
 
@@ -715,36 +735,35 @@ __global__ void probe_one_token_kernel(const T* __restrict__ q, float* __restric
   probe_kv[(size_t(unit) * n_kv_heads + g) * D + ch] = acc / float(group);
 }
 
-// Returns 1 when the shape does not suit the streaming kernel (the caller takes the cluster kernel).
+// The batched kernel: two CTAs per SM.  Returns 1 when the shape does not suit it (the caller takes the cluster kernel).
 template <typename T, int D>
-int launch_stream(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaStream_t st, int n_sm) {
+int launch_ring(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaStream_t st, int n_sm) {
   constexpr int VN = Vec16<T>::N;
-  constexpr int RL = kStreamThreads / (D / VN), NP = kStreamThreads / D;
+  constexpr int RL = kRingThreads / (D / VN), NW = kRingThreads / 32;
+  constexpr int kChunkRows = RL * kRingRowsPerThread;
   const int W = p.n_tokens;
-  const int per = std::max(1, (W + RL * kMaxChunks - 1) / (RL * kMaxChunks));
-  const int chunk_rows = RL * per, n_chunks = (W + chunk_rows - 1) / chunk_rows;
-  const size_t tile_bytes = (size_t(chunk_rows) * n_chunks * D * sizeof(T) + 127) & ~size_t(127);
-  const size_t smem = tile_bytes + sizeof(float) * (size_t(2) * (kStreamThreads / 32) * D + 2 * NP * D + 5 * D + 32 + ((W + 3) & ~3)) +
-                      8 * kMaxChunks;
-  if (smem > 227 * 1024) return 1;                    // the tile does not fit
-  if (chunk_rows > 256) return 1;                     // a box dimension holds at most 256
+  if (kChunkRows > 256) return 1;                     // a box dimension holds at most 256
+  const int n_chunks = (W + kChunkRows - 1) / kChunkRows;
+  const size_t smem = size_t(kRingSlots) * kChunkRows * D * sizeof(T) +
+                      sizeof(float) * (size_t(2) * NW * D + 6 * D + 32 + ((W + 3) & ~3)) + 8 * 2 * kRingSlots;
+  if (smem > 227 * 1024 / kRingCtasPerSm - 1024) return 1;      // kRingCtasPerSm CTAs must fit an SM
   CUtensorMap tm_q;
-  if (!encode_q<T, D>(&tm_q, p, b.units(), chunk_rows)) return ACTQKV_ERR_LAUNCH;
-  auto kern = bias_probe_stream_kernel<T, D>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-    return ACTQKV_ERR_LAUNCH;
+  if (!encode_q<T, D>(&tm_q, p, b.units(), kChunkRows)) return ACTQKV_ERR_LAUNCH;
+  auto kern = bias_probe_ring_kernel<T, D>;
+  static std::atomic<bool> opted_in[kMaxDevices];
+  if (!opt_in_shared_memory(kern, 227 * 1024 / kRingCtasPerSm - 1024, opted_in)) return ACTQKV_ERR_LAUNCH;
   prefer_max_shared(kern);
   const int n_items = b.units() * cfg->n_q_heads;
   cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(std::min(n_items, n_sm), 1, 1);
-  lc.blockDim = dim3(kStreamThreads, 1, 1);
+  lc.gridDim = dim3(std::min(n_items, kRingCtasPerSm * n_sm), 1, 1);
+  lc.blockDim = dim3(kRingThreads + 32, 1, 1);
   lc.dynamicSmemBytes = smem;
   lc.stream = st;
   cudaLaunchAttribute attr[1];
   allow_early_launch(attr[0]);
   lc.attrs = attr;
   lc.numAttrs = 1;
-  if (cudaLaunchKernelEx(&lc, kern, tm_q, p, n_items, chunk_rows, n_chunks) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&lc, kern, tm_q, p, n_items, n_chunks) != cudaSuccess) {
     (void)cudaGetLastError();
     return ACTQKV_ERR_LAUNCH;
   }
@@ -762,7 +781,7 @@ int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaS
   int dev = 0, n_sm = 0;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
   if (n_sm > 0 && b.units() * cfg->n_q_heads >= 2 * n_sm) {
-    const int rc = launch_stream<T, D>(cfg, b, p, st, n_sm);
+    const int rc = launch_ring<T, D>(cfg, b, p, st, n_sm);
     if (rc <= 0) return rc;
   }
   auto kern = bias_probe_kernel<T, D>;

@@ -227,6 +227,8 @@ __global__ void __launch_bounds__(32)
 entropy_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_cand,
                float* __restrict__ theta, int n_kv_heads, int n_cap, int n_layers, float beta) {
   const int g = blockIdx.x, unit = blockIdx.y;
+  grid_dependency_wait();            // the scores come from the stream's previous kernel
+  grid_launch_dependents();
   const int n = min(n_cand[unit / n_layers], n_cap);
   const float th = warp_entropy(scores + (size_t(unit) * n_kv_heads + g) * n_cap, n, beta);
   if (threadIdx.x == 0) theta[size_t(unit) * n_kv_heads + g] = th;
@@ -285,8 +287,17 @@ int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_k
 int launch_entropy(const actqkv_config* cfg, const Batch& b, const float* scores, const int32_t* n_cand,
                    float* theta, cudaStream_t st) {
   prefer_max_shared(entropy_kernel);
-  entropy_kernel<<<dim3(cfg->n_kv_heads, b.units()), 32, 0, st>>>(scores, n_cand, theta, cfg->n_kv_heads, cfg->n_cap,
-                                                                 b.n_layers, cfg->beta);
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(cfg->n_kv_heads, b.units(), 1);
+  lc.blockDim = dim3(32, 1, 1);
+  lc.stream = st;
+  cudaLaunchAttribute attr[1];
+  allow_early_launch(attr[0]);       // resident while the score kernel drains; waits for it before reading
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  if (cudaLaunchKernelEx(&lc, entropy_kernel, scores, n_cand, theta, cfg->n_kv_heads, cfg->n_cap, b.n_layers,
+                         cfg->beta) != cudaSuccess)
+    return ACTQKV_ERR_LAUNCH;
   return launch_status();
 }
 

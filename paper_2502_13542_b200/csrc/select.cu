@@ -56,6 +56,8 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
   extern __shared__ float theta_h[];   // [Lb][Hkv]
   const int seq = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  grid_dependency_wait();            // scores / densities come from the stream's previous kernels
+  grid_launch_dependents();
   const int n = min(p.n_cand[seq], p.n_cap);
   for (int pair = warp; pair < p.Lb * p.n_kv_heads; pair += kChainThreads / 32) {
     const size_t uh = size_t(seq) * p.Lb * p.n_kv_heads + pair;
@@ -371,8 +373,16 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
       p.theta_in = theta_out;
     }
     prefer_max_shared(cutoff_chain_kernel);
-    cutoff_chain_kernel<<<b.n_seq, kChainThreads, sm_chain, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return ACTQKV_ERR_LAUNCH;
+    cudaLaunchConfig_t lcc = {};
+    lcc.gridDim = dim3(b.n_seq, 1, 1);
+    lcc.blockDim = dim3(kChainThreads, 1, 1);
+    lcc.dynamicSmemBytes = sm_chain;
+    lcc.stream = st;
+    cudaLaunchAttribute cattr[1];
+    allow_early_launch(cattr[0]);
+    lcc.attrs = cattr;
+    lcc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lcc, cutoff_chain_kernel, p) != cudaSuccess) return ACTQKV_ERR_LAUNCH;
     if (cfg->cap_blocks == 0) return ACTQKV_OK;
   }
   prefer_max_shared(kern);
@@ -388,7 +398,7 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
   attr[0].val.clusterDim.z = 1;
   allow_early_launch(attr[1]);
   lc.attrs = attr;
-  lc.numAttrs = fused ? 2 : 1;      // after the chain kernel (plain launch) the selection starts normally
+  lc.numAttrs = 2;                  // every kernel of the chain waits for its predecessor before it reads
   if (cudaLaunchKernelEx(&lc, kern, scores, n_cand, sel_count, sel_idx, cfg->n_kv_heads, cfg->n_cap,
                          cfg->cap_blocks, b.n_layers, status, p) != cudaSuccess)
     return ACTQKV_ERR_LAUNCH;
