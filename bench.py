@@ -90,7 +90,7 @@ class ClockSampler(threading.Thread):
 # DRAM traffic of one launch of the attention kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
 # ncu capture of this workload), valid only for the kernel source it was taken on: the figure is
 # reported while the sha256 of the kernel file still starts with the recorded digits, else null.
-ATTENTION_TRAFFIC = {"source_sha256_16": "8f25a2402d12373f", "bytes_per_launch": 23673856}
+ATTENTION_TRAFFIC = {"source_sha256_16": "2029540e3952bb66", "bytes_per_launch": 23672064}
 
 
 def attention_traffic():
@@ -670,14 +670,14 @@ def _time_stage(fn, iters, flush):
     return 1e3 * t[len(t) // 2], 1e3 * t[0]          # median and minimum, microseconds
 
 
-def measure_stack32(iters, dev):
+def measure_stack32(iters, dev, n_layers=32):
     """All 32 layers of the LLaMA3-8B shape batched in one launch per stage at the last window of a
     32k prefill: Q = 134 MB, representative table = 66 MB per launch (larger than or comparable
     to L2; L2 is flushed before every timed launch)."""
     import torch
     from paper_2502_13542_b200 import binding as B
     from paper_2502_13542_b200 import workloads as wl
-    spec = wl.llama3_8b_stack32()
+    spec = wl.llama3_8b_stack32().replace(n_layers=n_layers)
     L = spec.n_layers
     cfg = B.make_config(spec, out_dtype=B.BF16)
     st = B.RetrievalState(cfg, n_seq=1, n_layers=L, page_table=wl.shuffled_page_table(spec, spec.context)[None, :], device=dev)
@@ -720,7 +720,7 @@ def measure_stack32(iters, dev):
         res[name] = {"us": us, "min_us": us_min, "bytes": nbytes, "GBps": nbytes / us / 1e3,
                      "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
     assert int(st.status.item()) == 0
-    return {"workload": "llama3_8b_stack32_32k: 32 layers batched per launch, last window", "stages": res,
+    return {"workload": f"llama3_8b_stack32_32k: {L} layers batched per launch, last window", "stages": res,
             "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
             "cold_l2": "512 MB read through L2 before every timed launch"}
 
@@ -930,6 +930,7 @@ def main():
     ap.add_argument("--workload", default="layer32k", choices=["layer32k", "stack32", "decode16", "long131k", "scorefull"],
                     help="layer32k = the headline line (which also carries the others' figures unless --headline-only); "
                          "the others print one secondary measurement alone")
+    ap.add_argument("--stack-layers", type=int, default=32, help="stack32 workload: layers batched per launch")
     ap.add_argument("--reps", type=int, default=20, help="repetitions of the timed K-step region (median reported)")
     ap.add_argument("--headline-only", action="store_true",
                     help="skip the secondary measurements (batched stages, 131k sweep, sustained loop)")
@@ -960,7 +961,7 @@ def main():
         dev = torch.device("cuda", 0)
         iters = args.steps if args.steps < 100 else 30
         if args.workload == "stack32":
-            print(json.dumps(measure_stack32(iters, dev)))
+            print(json.dumps(measure_stack32(iters, dev, args.stack_layers)))
         elif args.workload == "decode16":
             print(json.dumps(measure_decode16(iters, dev, args.decode_splits)))
         elif args.workload == "scorefull":
