@@ -180,27 +180,61 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   cluster_sync_all();         // both CTAs' barriers are initialised and both hold their TMEM
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  grid_dependency_wait();            // the selection (and whatever produced Q / K / V) is complete from here on
-  // ---- geometry (uniform over the CTA)
+  // ---- before the dependency wait: everything that does not depend on the selection.  The kernel
+  // launched just before this one may still be running (programmatic dependent launch), but every
+  // kernel of the library waits for its own predecessor before it lets its successor start, and none
+  // of those that do so writes the position, the page table, the cache pages of past tokens or the
+  // step's own Q / K / V: they are safe to read here.  Only sel_idx / sel_count must wait.
   const Geometry geo = make_geometry(p.a.pos0[seq], p.n_init, p.block, p.n_local_prev);
+  KeyStream ks;
+  ks.sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
+  ks.pt = p.a.page_table + size_t(seq) * p.max_pages;
+  ks.gpb = p.block / 16;                                 // page granules per block
+  ks.g_init = geo.init_len / 16;
+  ks.g_sel = 0;
+  ks.g_past = ks.g_init;                                 // for the early look-ups: the initial tokens only
+  ks.n_cand = geo.n_cand; ks.n_init = p.n_init; ks.block = p.block; ks.max_pages = p.max_pages;
+  ks.n_phys_pages = p.n_phys_pages; ks.page_base = layer_local * p.n_phys_pages;
+  ks.page_oob = p.n_layers * p.n_phys_pages;             // beyond the tensor: zero fill
+  ks.local_start = geo.local_start;
+  // Key tile 0 consists of initial tokens alone when there are at least 128 of them: its copies
+  // (and Q's) are issued now, so that the first S is ready right after the wait.
+  const bool early0 = !smem_short && geo.init_len >= kBN;
+  if ((warp == 0 || warp == 2) && !smem_short) {
+    const bool is_v = warp == 2;
+    if (!is_v && lane == 0) {
+      if (leader) mbar_expect_tx(bar_q, 2 * kTileBytes);
+      tma2_load_3d(q_smem, &tm_q, leader_addr(bar_q), 0, h, unit * nt + mt * kBM);
+      tma2_load_3d(q_smem + kSubTileBytes, &tm_q, leader_addr(bar_q), 64, h, unit * nt + mt * kBM);
+    }
+    if (early0) {
+      const int half = (lane >> 2) & 1, slot = lane & 3;
+      const int gi = is_v ? (lane & 7) : int(rank) * 4 + slot;
+      const int page = lane < 8 ? granule_page(ks, gi, p.a.status, !is_v && leader) : ks.page_oob;
+      const uint32_t full_local = is_v ? bar_vfull(0) : bar_kfull(0);
+      const uint32_t full = is_v ? full_local : leader_addr(full_local);
+      if (lane == 0) {
+        if (is_v) mbar_expect_tx(full_local, kHalfBytes);
+        else if (leader) mbar_expect_tx(full_local, kTileBytes);
+      }
+      __syncwarp();
+      if (lane < 8) {
+        if (is_v) tma_load_4d(v_ring + lane * 2048u, &tm_vp, full, int(rank) * 64, 0, g, page);
+        else tma2_load_4d(k_ring + half * kKSubBytes + slot * 2048u, &tm_kp, full, half * 64, 0, g, page);
+      }
+    }
+  }
+  grid_dependency_wait();            // the selection is complete from here on
+  // ---- geometry that depends on the selection (uniform over the CTA)
   int c = p.a.sel_count ? p.a.sel_count[unit] : 0;
   bool bad = false;
   if (c < 0 || c > p.cap_blocks || c > geo.n_cand) {
     bad = true;
     c = max(0, min(c, min(p.cap_blocks, geo.n_cand)));
   }
-  KeyStream ks;
-  ks.sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
-  ks.pt = p.a.page_table + size_t(seq) * p.max_pages;
-  ks.gpb = p.block / 16;                                 // page granules per block
-  ks.g_init = geo.init_len / 16;
   ks.g_sel = c * ks.gpb;
   const int64_t local_len = geo.p0 - geo.local_start;
   ks.g_past = ks.g_init + ks.g_sel + int((local_len + 15) / 16);   // the last local page may be partly filled
-  ks.n_cand = geo.n_cand; ks.n_init = p.n_init; ks.block = p.block; ks.max_pages = p.max_pages;
-  ks.n_phys_pages = p.n_phys_pages; ks.page_base = layer_local * p.n_phys_pages;
-  ks.page_oob = p.n_layers * p.n_phys_pages;             // beyond the tensor: zero fill
-  ks.local_start = geo.local_start;
   const bool misaligned = smem_short;
   const int n_past = geo.init_len + c * p.block + int(local_len);     // exact: the tail of the last page is masked
   const int past_tiles = (n_past + kBN - 1) / kBN;
@@ -222,11 +256,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t ring = is_v ? v_ring : k_ring;
     const CUtensorMap* tm_pages = is_v ? &tm_vp : &tm_kp;
     const CUtensorMap* tm_win = is_v ? &tm_vw : &tm_kw;
-    if (!is_v && lane == 0) {
-      if (leader) mbar_expect_tx(bar_q, 2 * kTileBytes);
-      tma2_load_3d(q_smem, &tm_q, leader_addr(bar_q), 0, h, unit * nt + mt * kBM);
-      tma2_load_3d(q_smem + kSubTileBytes, &tm_q, leader_addr(bar_q), 64, h, unit * nt + mt * kBM);
-    }
+    // (Q and, when it holds initial tokens only, tile 0 were issued before the dependency wait.)
     // lanes 0-7 issue one box each.  K: (channel half, granule 4 * rank + slot); V: granule = lane.
     const int half = (lane >> 2) & 1, slot = lane & 3;
     const int my_granule = is_v ? (lane & 7) : int(rank) * 4 + slot;
@@ -239,9 +269,11 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     };
     int page_cur = 0, page_next = resolve(0);
     bool ok = true;
-    int issued = 0;
+    const int j0 = early0 ? 1 : 0;
+    int issued = j0;
     const int ring_n = is_v ? kRingV : kRing;
-    for (int j = 0; j < n_tiles && ok; ++j) {
+    if (early0) page_cur = page_next;  // what the loop would have done at j = 0 besides the copies ...
+    for (int j = j0; j < n_tiles && ok; ++j) {
       const int s = j % ring_n, it = j / ring_n;
       if ((j & 3) == 0) page_cur = page_next;
       const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + my_granule);
@@ -272,7 +304,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
       }
       issued = j + 1;
-      if ((j & 3) == 0) page_next = resolve((j >> 2) + 1);   // after the issue: its stall is behind the ring
+      // the next chunk of look-ups after the issue: its stall is behind the ring (... and at j = 1 for tile 0's share)
+      if ((j & 3) == 0 || (early0 && j == 1)) page_next = resolve((j >> 2) + 1);
     }
     // drain: what this CTA issued must have landed before it may leave on the abort path; its
     // copies complete on the leader's barriers, which only the leader can poll, so the peer waits
