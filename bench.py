@@ -296,6 +296,21 @@ def run_ours(args):
     for i in range(args.warmup):
         one_step(i)
     barrier()
+    # The K steps of the timed region are captured once into a CUDA graph (the launch pattern of a
+    # prefill: one window through a run of layers, here the rotated layer states) and each
+    # repetition replays it: enqueueing a step's five launches from Python takes about as long as
+    # the step runs, so eager launches reach the GPU too late for the step's kernels to be
+    # resident ahead of their turn (programmatic dependent launch).  --eager times the plain
+    # launches instead.
+    step_graph = None
+    if not args.eager:
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(step_graph):
+            for i in range(args.steps):
+                one_step(args.warmup + i)
+        for _ in range(2):
+            step_graph.replay()
+        barrier()
     sampler = ClockSampler(local)
     sampler.start()
     if args.profile_region:
@@ -308,8 +323,11 @@ def run_ours(args):
         barrier()
         e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
-        for i in range(args.steps):
-            one_step(step_idx + i)
+        if step_graph is not None:
+            step_graph.replay()
+        else:
+            for i in range(args.steps):
+                one_step(step_idx + i)
         e1.record()
         step_idx += args.steps
         barrier()
@@ -506,7 +524,8 @@ def run_ours(args):
         "config": {"workload": "llama3_8b_layer_32k: last window (p0=32256) of a 32768-token prefill, "
                                "Hq=32 Hkv=8 D=128 W=512 B=128 r=4 n_init=128 k=cap=32, bf16 16-token pages",
                    "cold_l2": f"{n_copies} distinct layer-state copies rotated (inputs larger than L2)",
-                   "selected_blocks": c_sel, "parallelism": f"independent layers x{world}", "streams": "append on a second stream, joined every step"},
+                   "selected_blocks": c_sel, "parallelism": f"independent layers x{world}", "streams": "append on a second stream, joined every step",
+                   "launch": "eager calls" if args.eager else f"one CUDA graph of the {args.steps} steps, replayed per repetition"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps * len(rep_ms),
         "roofline": roofline, "stages": stages, "step_stats": step_stats,
     }
@@ -932,6 +951,8 @@ def main():
                          "the others print one secondary measurement alone")
     ap.add_argument("--stack-layers", type=int, default=32, help="stack32 workload: layers batched per launch")
     ap.add_argument("--reps", type=int, default=20, help="repetitions of the timed K-step region (median reported)")
+    ap.add_argument("--eager", action="store_true",
+                    help="enqueue the timed steps call by call from Python instead of replaying a CUDA graph of them")
     ap.add_argument("--headline-only", action="store_true",
                     help="skip the secondary measurements (batched stages, 131k sweep, sustained loop)")
     ap.add_argument("--decode-splits", type=int, default=1,

@@ -1,7 +1,10 @@
 // Step 5, tensor-core kernel for CTA pairs: the same attention as attention_tc.cu,
 //   [initial tokens | selected blocks | local past | window tokens (causal)]     (Eq. 2)
 // for bf16, D = 128, 16-token pages, with two CTAs (a cluster of 2, on two SMs) sharing every
-// K / V tile.
+// K / V tile.  The keys are visited in the order [initial | local past | window | selected]: all
+// but the selected blocks are known before this step's selection exists, so the kernel is launched
+// while the selection is still being computed (programmatic dependent launch), works through those
+// tiles, and takes the dependency wait only where the selected blocks begin.
 //
 // The single-CTA kernel streams a whole 64 KiB K+V tile into every CTA for 128 query rows and is
 // bound by that L2 -> shared-memory traffic.  Here the two CTAs of a pair hold the same 128 window
@@ -57,7 +60,7 @@ constexpr uint32_t kHalfBytes = kTileBytes / 2;          // 16 KiB: what one CTA
 constexpr uint32_t kKSubBytes = 64 * 128;                // [64 keys x 64 channels] sub-tile of a K half
 constexpr uint32_t kSmemTiles = kTileBytes + (kRing + kRingV) * kHalfBytes;
 constexpr int kFRing = 4;                                // O correction factors in flight
-constexpr int kNumBars = 1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + 2 * kFRing + 1;
+constexpr int kNumBars = 1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + 2 * kFRing + 2;
 constexpr uint32_t kBarBytes = 448;                      // barriers, TMEM slot, abort flag
 constexpr uint32_t kXchgBytes = (2 + kFRing) * 128 * 4;  // final row sums and maxima [row], O factors [ring][row]
 constexpr uint32_t kSmemNeeded = kSmemTiles + kBarBytes + kXchgBytes;
@@ -119,6 +122,39 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// ---------------------------------------------------------------- the paged key stream, in two parts
+struct PairKeys {
+  const int32_t* sel;
+  const int32_t* pt;
+  int g_init, g_a, g_b, gpb, n_cand, n_init, block, max_pages, n_phys_pages, page_base, page_oob;
+  int64_t local_page0;
+};
+// Row of the 4-D tensor map of logical page lp; page_oob (outside the tensor: TMA fills zeros) for
+// rejected table entries.
+__device__ __forceinline__ int physical_page(const PairKeys& ks, int64_t lp, int32_t* status, bool report) {
+  const int phys = lp < ks.max_pages ? ks.pt[lp] : -1;
+  if (phys < 0 || phys >= ks.n_phys_pages) {
+    if (report) set_status(status, ACTQKV_DEV_BAD_PAGE);
+    return ks.page_oob;
+  }
+  return ks.page_base + phys;
+}
+// Part A, 16-token granule gi: the initial tokens, then the local past up to p0.
+__device__ __forceinline__ int page_a(const PairKeys& ks, int gi, int32_t* status, bool report) {
+  if (gi >= ks.g_a) return ks.page_oob;
+  return physical_page(ks, gi < ks.g_init ? int64_t(gi) : ks.local_page0 + (gi - ks.g_init), status, report);
+}
+// Part B, granule gi: the selected blocks in the order of sel_idx.
+__device__ __forceinline__ int page_b(const PairKeys& ks, int gi, int32_t* status, bool report) {
+  if (gi >= ks.g_b) return ks.page_oob;
+  const int blk = ks.sel[gi / ks.gpb];
+  if (blk < 0 || blk >= ks.n_cand) {
+    if (report) set_status(status, ACTQKV_DEV_BAD_SELECTION);
+    return ks.page_oob;
+  }
+  return physical_page(ks, (int64_t(ks.n_init) + int64_t(blk) * ks.block) / 16 + gi % ks.gpb, status, report);
+}
+
 // ---------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kw,
@@ -144,7 +180,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   auto bar_vready = [&](int s) { return bars + 8u * (1 + 2 * kRing + 2 * kRingV + 2 * kSBuf + kPvRing + s); };
   auto bar_f = [&](int i) { return bars + 8u * (1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + i); };
   auto bar_corr = [&](int i) { return bars + 8u * (1 + 2 * kRing + 3 * kRingV + 2 * kSBuf + kPvRing + kFRing + i); };
-  const uint32_t bar_done = bars + 8u * (kNumBars - 1);
+  const uint32_t bar_done = bars + 8u * (kNumBars - 2);
+  const uint32_t bar_sel = bars + 8u * (kNumBars - 1);      // the selection has arrived (this CTA's K producer)
   unsigned char* base_generic = smem_raw + (base - raw);
   unsigned char* bars_generic = base_generic + kSmemTiles;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_generic + 8 * kNumBars);
@@ -153,7 +190,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   float* m_share = l_share + 128;                                        // [128] running maxima, for the log-sum-exp
   float* f_share = m_share + 128;                                        // [kFRing][128] O correction factors
 
-  const int h = blockIdx.x, mt = blockIdx.y, unit = blockIdx.z;      // the pair = heads (h & ~1, h | 1)
+  // the query tiles with the most keys (the last of the window) are launched first
+  const int h = blockIdx.x, mt = int(gridDim.y) - 1 - int(blockIdx.y), unit = blockIdx.z;      // the pair = heads (h & ~1, h | 1)
   const uint32_t rank = cluster_rank();                               // 0 = leader
   const bool leader = rank == 0;
   const int g = h / p.group, seq = unit / p.n_layers, layer_local = unit - seq * p.n_layers;
@@ -169,6 +207,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     for (int i = 0; i < kPvRing; ++i) mbar_init(bar_pvdone(i), 1);
     for (int i = 0; i < kFRing; ++i) { mbar_init(bar_f(i), kSoftmaxWarps); mbar_init(bar_corr(i), 8); }
     mbar_init(bar_done, 1);
+    mbar_init(bar_sel, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -180,68 +219,47 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   cluster_sync_all();         // both CTAs' barriers are initialised and both hold their TMEM
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  // ---- before the dependency wait: everything that does not depend on the selection.  The kernel
-  // launched just before this one may still be running (programmatic dependent launch), but every
-  // kernel of the library waits for its own predecessor before it lets its successor start, and none
-  // of those that do so writes the position, the page table, the cache pages of past tokens or the
-  // step's own Q / K / V: they are safe to read here.  Only sel_idx / sel_count must wait.
+  // ---- the key stream in two parts.  Part A needs nothing of this step's selection: the initial
+  // tokens and the local past (one run of 16-token pages, a ragged last tile masked), then the
+  // window's own tiles (causal on the last).  Part B, the selected blocks, follows the dependency
+  // wait.  The softmax is running, so the order of the tiles changes the rounding only.  The kernel
+  // launched just before this one may still be running while part A is worked on (programmatic
+  // dependent launch): every kernel of the library waits for its own predecessor before it writes,
+  // and none of those that let their successor start early writes the position, the page table,
+  // the cache pages of past tokens or the step's own Q / K / V.  Only sel_idx / sel_count must wait.
   const Geometry geo = make_geometry(p.a.pos0[seq], p.n_init, p.block, p.n_local_prev);
-  KeyStream ks;
+  const int64_t local_len = geo.p0 - geo.local_start;
+  PairKeys ks;
   ks.sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
   ks.pt = p.a.page_table + size_t(seq) * p.max_pages;
   ks.gpb = p.block / 16;                                 // page granules per block
   ks.g_init = geo.init_len / 16;
-  ks.g_sel = 0;
-  ks.g_past = ks.g_init;                                 // for the early look-ups: the initial tokens only
+  ks.g_a = ks.g_init + int((local_len + 15) / 16);       // the last local page may be partly filled
+  ks.g_b = 0;
+  ks.local_page0 = geo.local_start / 16;
   ks.n_cand = geo.n_cand; ks.n_init = p.n_init; ks.block = p.block; ks.max_pages = p.max_pages;
   ks.n_phys_pages = p.n_phys_pages; ks.page_base = layer_local * p.n_phys_pages;
   ks.page_oob = p.n_layers * p.n_phys_pages;             // beyond the tensor: zero fill
-  ks.local_start = geo.local_start;
-  // Key tile 0 consists of initial tokens alone when there are at least 128 of them: its copies
-  // (and Q's) are issued now, so that the first S is ready right after the wait.
-  const bool early0 = !smem_short && geo.init_len >= kBN;
-  if ((warp == 0 || warp == 2) && !smem_short) {
-    const bool is_v = warp == 2;
-    if (!is_v && lane == 0) {
-      if (leader) mbar_expect_tx(bar_q, 2 * kTileBytes);
-      tma2_load_3d(q_smem, &tm_q, leader_addr(bar_q), 0, h, unit * nt + mt * kBM);
-      tma2_load_3d(q_smem + kSubTileBytes, &tm_q, leader_addr(bar_q), 64, h, unit * nt + mt * kBM);
+  const int n_a = geo.init_len + int(local_len);         // exact: the tail of the last page is masked
+  const int tiles_a = (n_a + kBN - 1) / kBN;
+  const int n1 = tiles_a + mt + 1;                       // tiles before the dependency wait
+  int n_b = 0;                                           // keys of the selected blocks, known after the wait
+  // Every thread that needs the total takes the wait itself (it is the launch dependency, so it
+  // always ends) and reads the count: no role then waits on another one for it.
+  auto total_after_wait = [&](bool report) -> int {
+    grid_dependency_wait();            // the selection is complete from here on
+    int c = p.a.sel_count ? p.a.sel_count[unit] : 0;
+    if (c < 0 || c > p.cap_blocks || c > geo.n_cand) {
+      if (report) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
+      c = max(0, min(c, min(p.cap_blocks, geo.n_cand)));
     }
-    if (early0) {
-      const int half = (lane >> 2) & 1, slot = lane & 3;
-      const int gi = is_v ? (lane & 7) : int(rank) * 4 + slot;
-      const int page = lane < 8 ? granule_page(ks, gi, p.a.status, !is_v && leader) : ks.page_oob;
-      const uint32_t full_local = is_v ? bar_vfull(0) : bar_kfull(0);
-      const uint32_t full = is_v ? full_local : leader_addr(full_local);
-      if (lane == 0) {
-        if (is_v) mbar_expect_tx(full_local, kHalfBytes);
-        else if (leader) mbar_expect_tx(full_local, kTileBytes);
-      }
-      __syncwarp();
-      if (lane < 8) {
-        if (is_v) tma_load_4d(v_ring + lane * 2048u, &tm_vp, full, int(rank) * 64, 0, g, page);
-        else tma2_load_4d(k_ring + half * kKSubBytes + slot * 2048u, &tm_kp, full, half * 64, 0, g, page);
-      }
-    }
-  }
-  grid_dependency_wait();            // the selection is complete from here on
-  // ---- geometry that depends on the selection (uniform over the CTA)
-  int c = p.a.sel_count ? p.a.sel_count[unit] : 0;
-  bool bad = false;
-  if (c < 0 || c > p.cap_blocks || c > geo.n_cand) {
-    bad = true;
-    c = max(0, min(c, min(p.cap_blocks, geo.n_cand)));
-  }
-  ks.g_sel = c * ks.gpb;
-  const int64_t local_len = geo.p0 - geo.local_start;
-  ks.g_past = ks.g_init + ks.g_sel + int((local_len + 15) / 16);   // the last local page may be partly filled
-  const bool misaligned = smem_short;
-  const int n_past = geo.init_len + c * p.block + int(local_len);     // exact: the tail of the last page is masked
-  const int past_tiles = (n_past + kBN - 1) / kBN;
-  const int n_tiles = past_tiles + mt + 1;
+    n_b = c * p.block;
+    ks.g_b = c * ks.gpb;
+    return n1 + (n_b + kBN - 1) / kBN;
+  };
 
-  if (tid == 0 && (bad || misaligned)) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
-  if (misaligned) {           // uniform over the pair: nothing was issued yet
+  if (smem_short) {           // uniform over the pair: nothing was issued yet
+    if (tid == 0) set_status(p.a.status, ACTQKV_DEV_BAD_SELECTION);
     cluster_sync_all();
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
     return;
@@ -250,62 +268,77 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   if (warp == 0 || warp == 2) {
     // =========================== TMA producers: warp 0 -> K half (and Q), warp 2 -> V half ===========================
     // This CTA's half of a tile: keys [64 * rank, +64) of K (all channels), channels [64 * rank, +64)
-    // of V (all keys).  Copies complete on the leader's barriers; the leader posts the byte count
-    // of both halves.
+    // of V (all keys).  K copies complete on the leader's barriers (the leader posts the byte count
+    // of both halves), a V half on its own CTA's barrier, where that CTA's converter warps pick it up.
     const bool is_v = warp == 2;
     const uint32_t ring = is_v ? v_ring : k_ring;
     const CUtensorMap* tm_pages = is_v ? &tm_vp : &tm_kp;
     const CUtensorMap* tm_win = is_v ? &tm_vw : &tm_kw;
-    // (Q and, when it holds initial tokens only, tile 0 were issued before the dependency wait.)
+    const int ring_n = is_v ? kRingV : kRing;
+    if (!is_v && lane == 0) {
+      if (leader) mbar_expect_tx(bar_q, 2 * kTileBytes);
+      tma2_load_3d(q_smem, &tm_q, leader_addr(bar_q), 0, h, unit * nt + mt * kBM);
+      tma2_load_3d(q_smem + kSubTileBytes, &tm_q, leader_addr(bar_q), 64, h, unit * nt + mt * kBM);
+    }
     // lanes 0-7 issue one box each.  K: (channel half, granule 4 * rank + slot); V: granule = lane.
     const int half = (lane >> 2) & 1, slot = lane & 3;
     const int my_granule = is_v ? (lane & 7) : int(rank) * 4 + slot;
-    // Page lookups (sel_idx -> page_table, two dependent loads) are taken 32 granules = 4 tiles at
-    // a time, one granule per lane, one chunk ahead of the tiles being issued, so their latency
-    // is off the per-tile path; the issuing lane fetches its page with a shuffle.
-    auto resolve = [&](int chunk) {
-      const int gi = chunk * 32 + lane;
-      return gi < past_tiles * 8 ? granule_page(ks, gi, p.a.status, !is_v && leader) : ks.page_oob;
-    };
-    int page_cur = 0, page_next = resolve(0);
+    const bool report = !is_v && leader;
     bool ok = true;
-    const int j0 = early0 ? 1 : 0;
-    int issued = j0;
-    const int ring_n = is_v ? kRingV : kRing;
-    if (early0) page_cur = page_next;  // what the loop would have done at j = 0 besides the copies ...
-    for (int j = j0; j < n_tiles && ok; ++j) {
+    int issued = 0;
+    // waits for the ring slot of tile j and posts the bytes to come; returns the slot's base address
+    auto claim = [&](int j, uint32_t& full) -> uint32_t {
       const int s = j % ring_n, it = j / ring_n;
-      if ((j & 3) == 0) page_cur = page_next;
-      const int page = __shfl_sync(0xffffffffu, page_cur, (j & 3) * 8 + my_granule);
       if (it > 0) ok = mbar_wait(is_v ? bar_vempty(s) : bar_kempty(s), (it - 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      // K halves complete on the leader's barrier (the leader posts both halves' bytes); a V half
-      // completes on its own CTA's barrier, where that CTA's softmax threads pick it up
+      if (!ok) return 0;
       const uint32_t full_local = is_v ? bar_vfull(s) : bar_kfull(s);
-      const uint32_t full = is_v ? full_local : leader_addr(full_local);
-      const uint32_t sbase = ring + s * kHalfBytes;
+      full = is_v ? full_local : leader_addr(full_local);
       if (lane == 0) {
         if (is_v) mbar_expect_tx(full_local, kHalfBytes);
         else if (leader) mbar_expect_tx(full_local, kTileBytes);
       }
       __syncwarp();
-      if (j < past_tiles) {
+      return ring + s * kHalfBytes;
+    };
+    // `cnt` tiles of cache pages from tile j_base on.  Page look-ups (for part B sel_idx ->
+    // page_table, two dependent loads) are taken 32 granules = 4 tiles at a time, one granule per
+    // lane, one chunk ahead of the tiles being issued, so that their latency is off the per-tile
+    // path; the issuing lane fetches its page with a shuffle.
+    auto paged_tiles = [&](int j_base, int cnt, auto&& page_of) {
+      int page_cur = 0, page_next = page_of(lane);
+      for (int t = 0; t < cnt && ok; ++t) {
+        if ((t & 3) == 0) page_cur = page_next;
+        const int page = __shfl_sync(0xffffffffu, page_cur, (t & 3) * 8 + my_granule);
+        uint32_t full = 0;
+        const uint32_t sbase = claim(j_base + t, full);
+        if (!ok) break;
         if (lane < 8) {
           if (is_v) tma_load_4d(sbase + lane * 2048u, tm_pages, full, int(rank) * 64, 0, g, page);
           else tma2_load_4d(sbase + half * kKSubBytes + slot * 2048u, tm_pages, full, half * 64, 0, g, page);
         }
-      } else {
-        const int row0 = unit * nt + (j - past_tiles) * kBN;
-        if (is_v) {
-          if (lane == 0) tma_load_3d(sbase, tm_win, full, int(rank) * 64, g, row0);
-        } else if (lane < 2) {
-          tma2_load_3d(sbase + lane * kKSubBytes, tm_win, full, lane * 64, g, row0 + int(rank) * 64);
-        }
+        issued = j_base + t + 1;
+        // the next chunk of look-ups after the issue: its stall is behind the ring
+        if ((t & 3) == 0) page_next = page_of(((t >> 2) + 1) * 32 + lane);
       }
-      issued = j + 1;
-      // the next chunk of look-ups after the issue: its stall is behind the ring (... and at j = 1 for tile 0's share)
-      if ((j & 3) == 0 || (early0 && j == 1)) page_next = resolve((j >> 2) + 1);
+    };
+    paged_tiles(0, tiles_a, [&](int gi) { return page_a(ks, gi, p.a.status, report); });
+    for (int w = 0; w <= mt && ok; ++w) {
+      uint32_t full = 0;
+      const uint32_t sbase = claim(tiles_a + w, full);
+      if (!ok) break;
+      const int row0 = unit * nt + w * kBN;
+      if (is_v) {
+        if (lane == 0) tma_load_3d(sbase, tm_win, full, int(rank) * 64, g, row0);
+      } else if (lane < 2) {
+        tma2_load_3d(sbase + lane * kKSubBytes, tm_win, full, lane * 64, g, row0 + int(rank) * 64);
+      }
+      issued = tiles_a + w + 1;
+    }
+    if (ok) {
+      const int n_tiles = total_after_wait(report && lane == 0);
+      if (!is_v && lane == 0) mbar_arrive(bar_sel);      // the converter warps poll this instead of blocking
+      paged_tiles(n1, n_tiles - n1, [&](int gi) { return page_b(ks, gi, p.a.status, report); });
     }
     // drain: what this CTA issued must have landed before it may leave on the abort path; its
     // copies complete on the leader's barriers, which only the leader can poll, so the peer waits
@@ -335,7 +368,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         constexpr uint32_t idesc_qk = make_idesc(false, 2 * kBM, kBN);
         const uint32_t q_lo = desc_lo(q_smem, 16u);
         ok = mbar_wait(bar_q, 0, abort_flag);
-        for (int j = 0; j < n_tiles && ok; ++j) {
+        int n_tiles = n1;
+        for (int j = 0; ok; ++j) {
+          if (j == n1) n_tiles = total_after_wait(false);
+          if (j >= n_tiles) break;
           const int s = j % kRing;
           if (j >= kSBuf) ok = mbar_wait(bar_pvdone((j - kSBuf) % kPvRing), ((j - kSBuf) / kPvRing) & 1, abort_flag);
           ok = ok && mbar_wait(bar_kfull(s), (j / kRing) & 1, abort_flag);
@@ -358,7 +394,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       } else {
         constexpr uint32_t idesc_pv = make_idesc_f16(true, 2 * kBM, kBN);
         const uint32_t tmem_o = tmem + kSBuf * 128;
-        for (int i = 0; i < n_tiles && ok; ++i) {
+        int n_tiles = n1;
+        for (int i = 0; ok; ++i) {
+          if (i == n1) n_tiles = total_after_wait(false);
+          if (i >= n_tiles) break;
           const int s = i % kRingV, b = i % kSBuf;
           // P(i) published by every softmax warp of both CTAs, which also turned V(i) into fp16
           ok = mbar_wait(bar_vready(s), (i / kRingV) & 1, abort_flag);          // V(i) is fp16 in both CTAs
@@ -391,10 +430,25 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t o_row = tmem + (uint32_t(q4 * 32) << 16) + kSBuf * 128;
     constexpr int kLag = 2;                               // V is converted this many tiles ahead of the correction
     bool ok = true;
-    for (int it = 0; it < n_tiles + kLag && ok; ++it) {
-      if (it < n_tiles) {
-        const int vs = it % kRingV;
-        ok = mbar_wait(bar_vfull(vs), (it / kRingV) & 1, abort_flag);
+    // ci: next tile to convert, ri: next tile whose O correction is due.  Conversions lead by kLag.
+    // Where part A ends the total is not known yet: the K producer signals the arrival of the
+    // selection, and these warps only poll that signal while corrections of part A are still due
+    // (a blocking wait here would hold back the last products of part A).
+    int ci = 0, ri = 0, known = n1;
+    bool final = false;
+    while (ok) {
+      if (!final && ci >= known) {
+        bool ready = ri >= known || mbar_test_wait(bar_sel, 0);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {
+          known = total_after_wait(false);
+          final = true;
+        }
+      }
+      if (ri >= known) break;                             // only once the total is final
+      if (ci < known && ci <= ri + kLag) {
+        const int vs = ci % kRingV;
+        ok = mbar_wait(bar_vfull(vs), (ci / kRingV) & 1, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         uint4* vp = reinterpret_cast<uint4*>(base_generic + (v_ring - base) + vs * kHalfBytes);
@@ -406,9 +460,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core's reads
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_addr(bar_vready(vs)));
-      }
-      const int j = it - kLag;
-      if (j >= 0) {
+        ++ci;
+      } else {
+        const int j = ri;
         // The running maximum of tile j is known: where it grew, O (on the old maximum) is scaled
         // down before P(j) V(j) is added.  The softmax threads do not wait for this.
         ok = mbar_wait(bar_f(j % kFRing), (j / kFRing) & 1, abort_flag);
@@ -434,6 +488,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         }
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_addr(bar_corr(j % kFRing)));
+        ++ri;
       }
     }
   } else if (warp >= 4) {
@@ -452,7 +507,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t lane16 = uint32_t(q4 * 32 + hw * 16) << 16;
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;     // running maxima (log2 units) and partial row sums
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
+    int n_tiles = n1;
+    for (int j = 0;; ++j) {
+      if (j == n1) n_tiles = total_after_wait(false);
+      if (j >= n_tiles) break;
       const int sb = j % kSBuf;
       ok = mbar_wait(bar_sfull(sb), (j / kSBuf) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -463,9 +521,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       TMEM_LD16X256P_WAIT(s_addr, sv);
       // key-validity limits: ragged last past tile, or the causal diagonal of the last tile
       int lim0 = kBN, lim1 = kBN;
-      if (j < past_tiles) lim0 = lim1 = min(kBN, n_past - j * kBN);
-      else if (j == n_tiles - 1) { lim0 = row0 + 1; lim1 = row1 + 1; }
-      const bool masked = (j == n_tiles - 1) || (j == past_tiles - 1 && (n_past % kBN) != 0);   // CTA-uniform
+      if (j < tiles_a) lim0 = lim1 = min(kBN, n_a - j * kBN);
+      else if (j == n1 - 1) { lim0 = row0 + 1; lim1 = row1 + 1; }
+      else if (j >= n1) lim0 = lim1 = min(kBN, n_b - (j - n1) * kBN);
+      const bool masked = j == n1 - 1 || lim0 < kBN;      // CTA-uniform
       float mx0 = -INFINITY, mx1 = -INFINITY;
       if (masked) {
 #pragma unroll

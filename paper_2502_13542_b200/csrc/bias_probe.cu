@@ -83,8 +83,8 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
   const size_t hd = (size_t(unit) * p.n_q_heads + h) * D;
   const size_t uh = size_t(unit) * p.n_q_heads + h;
 
-  grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
   grid_launch_dependents();
+  grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
   // ---- 0. rows -> shared memory
   constexpr uint32_t kRowBytes = D * sizeof(T);
   const uint32_t bar_addr = smem_addr(bar);
@@ -415,8 +415,8 @@ bias_probe_ring_kernel(const __grid_constant__ CUtensorMap tm_q, BiasProbeParams
   const bool running = p.do_bias && p.stats_mode == ACTQKV_STATS_CUMULATIVE;
   const int n_pass = p.do_bias ? 2 : 1;
 
-  grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
   grid_launch_dependents();
+  grid_dependency_wait();            // q and the running statistics may come from earlier kernels of the stream
   if (tid == 0) {
     for (int s = 0; s < kRingSlots; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(bar_full + s)));

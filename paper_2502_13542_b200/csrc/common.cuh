@@ -62,10 +62,19 @@ inline void prefer_max_shared(Kernel kern) {
   (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, int(cudaSharedmemCarveoutMaxShared));
 }
 
-// Programmatic dependent launch: a kernel launched with this attribute may start (run its
-// prologue: barrier set-up, loads of inputs no earlier kernel of the stream writes) while the
-// kernel before it in the stream is still draining; it must execute grid_dependency_wait()
-// before it touches anything an earlier kernel writes.  Without the attribute the wait is a no-op.
+// Programmatic dependent launch: a kernel launched with this attribute may start while the kernel
+// before it in the stream is still running, as soon as every CTA of that kernel has executed
+// grid_launch_dependents() (or has left).  It must execute grid_dependency_wait() -- which returns
+// once the kernel before it has completed and its writes are visible -- before it WRITES anything
+// and before it reads anything that a kernel of the library writes.  The short kernels of a step
+// (bias + probe, score, density, cut-off, selection) let their successor start at once and wait
+// right after, so the whole chain of a step is resident early and each link starts the moment its
+// predecessor ends; since every link waits for its predecessor before it writes, the wait of the
+// last link still orders it after all of them.  What a kernel does BEFORE its wait may therefore
+// overlap any earlier kernel of the chain: it may read only what none of them writes (the step's
+// Q / K / V, positions, the page table, cache pages and table rows of past tokens).  Kernels that
+// write those (the append) neither start early nor let their successor start before they end.
+// Without the attribute the wait is a no-op.
 inline void allow_early_launch(cudaLaunchAttribute& a) {
   a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   a.val.programmaticStreamSerializationAllowed = 1;
@@ -94,7 +103,7 @@ inline int launch_status() { return cudaGetLastError() == cudaSuccess ? ACTQKV_O
 
 // ---------------------------------------------------------------- device helpers
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// Lets the next kernel of the stream start its prologue; called after this kernel's own wait.
+// Lets the next kernel of the stream become resident (it still waits for this one to end).
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void set_status(int32_t* status, int bit) {

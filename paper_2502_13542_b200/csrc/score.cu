@@ -86,8 +86,8 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
   Raw ra, rb;
   const bool first_fast = fast_shape && full(0);
   if (first_fast) load_fast(b0, ra); else load_group(b0, ga);
-  grid_dependency_wait();            // the table is older than the stream's previous kernel; the probe is not
   grid_launch_dependents();
+  grid_dependency_wait();            // the table is older than the stream's previous kernel; the probe is not
   const float* pg = probe_kv + (size_t(unit) * n_kv_heads + g) * D;
   float pv[VN];
   Vec16<float>::load_nc(pg + lir * VN, reinterpret_cast<float(&)[4]>(pv[0]));
@@ -227,8 +227,8 @@ __global__ void __launch_bounds__(32)
 entropy_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_cand,
                float* __restrict__ theta, int n_kv_heads, int n_cap, int n_layers, float beta) {
   const int g = blockIdx.x, unit = blockIdx.y;
-  grid_dependency_wait();            // the scores come from the stream's previous kernel
   grid_launch_dependents();
+  grid_dependency_wait();            // the scores come from the stream's previous kernel
   const int n = min(n_cand[unit / n_layers], n_cap);
   const float th = warp_entropy(scores + (size_t(unit) * n_kv_heads + g) * n_cap, n, beta);
   if (threadIdx.x == 0) theta[size_t(unit) * n_kv_heads + g] = th;

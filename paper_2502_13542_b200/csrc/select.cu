@@ -26,6 +26,7 @@ namespace {
 
 constexpr int kChainThreads = 1024;
 constexpr int kSelThreads = 256;
+constexpr int kRestCap = 128;          // deeper layers whose mean densities are divided out in parallel
 
 struct ChainParams {
   const float* scores;
@@ -56,8 +57,8 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
   extern __shared__ float theta_h[];   // [Lb][Hkv]
   const int seq = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  grid_dependency_wait();            // scores / densities come from the stream's previous kernels
   grid_launch_dependents();
+  grid_dependency_wait();            // scores / densities come from the stream's previous kernels
   const int n = min(p.n_cand[seq], p.n_cap);
   for (int pair = warp; pair < p.Lb * p.n_kv_heads; pair += kChainThreads / 32) {
     const size_t uh = size_t(seq) * p.Lb * p.n_kv_heads + pair;
@@ -183,33 +184,64 @@ __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_cand,
               int32_t* __restrict__ sel_count, int32_t* __restrict__ sel_idx, int n_kv_heads,
               int n_cap, int cap_blocks, int n_layers, int32_t* status, ChainParams ch) {
-  extern __shared__ uint32_t keys[];           // [n_cap]
+  extern __shared__ uint32_t sel_smem[];       // the head's scores [n_cap] (fp32), then their keys [n_cap]
+  float* sc = reinterpret_cast<float*>(sel_smem);
+  uint32_t* keys = sel_smem + n_cap;
+  __shared__ unsigned long long key64[kSelThreads];
   __shared__ int hist[256];
   __shared__ int warp_tot[kSelThreads / 32];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_need;
   __shared__ float sh_theta;                   // this head's density (read by the cluster peers)
   __shared__ int sh_count;
+  __shared__ double rest_q[kRestCap];          // mean density of each deeper layer with a history
+  __shared__ unsigned char rest_has[kRestCap];
+  __shared__ double sh_brem, sh_rest;
+  __shared__ int sh_no_hist;
   const int g = blockIdx.x, unit = blockIdx.y, tid = threadIdx.x;
-  grid_dependency_wait();            // scores / densities / counts come from the stream's previous kernels
   grid_launch_dependents();
+  grid_dependency_wait();            // scores / densities / counts come from the stream's previous kernels
   const int n = min(n_cand[unit / n_layers], n_cap);
   const float* s = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
+  // the scores are fetched once, by all threads at a time; density and selection read them from here
+  for (int i = tid; i < n; i += kSelThreads) sc[i] = s[i];
   int c;
   if constexpr (kFused) {
     cg::cluster_group cluster = cg::this_cluster();
     const int seq = unit;                      // one layer per call: unit == sequence
     const int layer = ch.layer0;
     double* st = ch.state + size_t(seq) * (1 + 2 * ch.L);
-    // the old state is read by every CTA before the cluster barrier, written by CTA 0 after it
-    double b_rem = 0.0, rest_hist = 0.0;
-    int no_hist = 0;
-    if (tid == 0) {
-      b_rem = layer == 0 ? double(ch.L) * double(ch.k_blocks) : st[0];
-      for (int j = layer + 1; j < ch.L; ++j) {
+    // The old state is read by every CTA before the cluster barrier, written by CTA 0 after it.
+    // The deeper layers' mean densities are divided out by one thread per layer; thread 32 then
+    // adds them in layer order (the order of the serial loop, so the sum has the same bits) while
+    // warp 0 takes this head's density.
+    const int deeper = ch.L - (layer + 1);
+    const bool spread = deeper <= kRestCap;
+    if (spread && tid >= 32) {
+      for (int t = tid - 32; t < deeper; t += kSelThreads - 32) {
+        const int j = layer + 1 + t;
         const double cnt = st[1 + ch.L + j];
-        if (cnt > 0.0) rest_hist += st[1 + j] / cnt; else ++no_hist;
+        rest_has[t] = cnt > 0.0;
+        rest_q[t] = cnt > 0.0 ? st[1 + j] / cnt : 0.0;
       }
+    }
+    __syncthreads();
+    if (tid == 32) {
+      double rest_hist = 0.0;
+      int no_hist = 0;
+      if (spread) {
+        for (int t = 0; t < deeper; ++t) {
+          if (rest_has[t]) rest_hist += rest_q[t]; else ++no_hist;
+        }
+      } else {
+        for (int j = layer + 1; j < ch.L; ++j) {
+          const double cnt = st[1 + ch.L + j];
+          if (cnt > 0.0) rest_hist += st[1 + j] / cnt; else ++no_hist;
+        }
+      }
+      sh_brem = layer == 0 ? double(ch.L) * double(ch.k_blocks) : st[0];
+      sh_rest = rest_hist;
+      sh_no_hist = no_hist;
     }
     if (tid < 32) {
       const size_t uh = size_t(unit) * n_kv_heads + g;
@@ -217,7 +249,7 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
       if (ch.theta_in) {
         th = ch.theta_in[uh];
       } else {
-        th = warp_entropy(s, n, ch.beta);
+        th = warp_entropy(sc, n, ch.beta);
         if (tid == 0 && ch.theta_out) ch.theta_out[uh] = th;
       }
       if (tid == 0) sh_theta = th;
@@ -232,6 +264,8 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
 #pragma unroll
       for (int h2 = 0; h2 < 8; ++h2) sum += double(th_h[h2]);
       const double th = sum / double(n_kv_heads);
+      const double b_rem = sh_brem, rest_hist = sh_rest;
+      const int no_hist = sh_no_hist;
       Grant gr{0, 0.0};
       if (n > 0) {
         // layers without history count with this layer's density; with every layer in the call
@@ -265,8 +299,23 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
   for (int i = c + tid; i < cap_blocks; i += kSelThreads) out[i] = -1;
   if (c >= n) {
     for (int i = tid; i < min(n, c); i += kSelThreads) out[i] = i;
+  } else if (c > 0 && n <= kSelThreads) {
+    // One candidate per thread: its rank is the number of candidates that come before it in the
+    // order (higher key first, equal keys by lower index), counted against all of them; the c
+    // first are taken and compacted in ascending index order.
+    const uint32_t k = tid < n ? score_key(sc[tid]) : 0u;
+    key64[tid] = tid < n ? ((static_cast<unsigned long long>(k) << 32) | uint32_t(~uint32_t(tid))) : 0ull;
+    __syncthreads();
+    const unsigned long long mine = key64[tid];
+    int rank = 0;
+#pragma unroll 4
+    for (int j = 0; j < n; ++j) rank += key64[j] > mine;
+    const int take = tid < n && rank < c;
+    int tot;
+    const int pos = block_exclusive_scan(take, warp_tot, &tot);
+    if (take && pos < cap_blocks) out[pos] = tid;
   } else if (c > 0) {
-    for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(s[i]);
+    for (int i = tid; i < n; i += kSelThreads) keys[i] = score_key(sc[i]);
     if (tid == 0) { sh_prefix = 0u; sh_need = c; }
     __syncthreads();
 
@@ -348,7 +397,7 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
                   int32_t* sel_count, float* budget_real, int32_t* status, cudaStream_t st) {
   if (cfg->thetabar_mode == ACTQKV_THETABAR_ALG1 && (b.layer0 != 0 || b.n_layers != cfg->n_layers))
     return ACTQKV_ERR_UNSUPPORTED;
-  if (size_t(cfg->n_cap) * 4 > 160 * 1024) return ACTQKV_ERR_SHAPE;
+  if (size_t(cfg->n_cap) * 8 > 200 * 1024) return ACTQKV_ERR_SHAPE;
   ChainParams p;
   p.scores = scores; p.theta_in = theta_in; p.theta_out = theta_out; p.n_cand = n_cand;
   p.state = static_cast<double*>(budget_state);
@@ -356,7 +405,7 @@ int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores,
   p.n_kv_heads = cfg->n_kv_heads; p.n_cap = cfg->n_cap; p.L = cfg->n_layers; p.Lb = b.n_layers;
   p.layer0 = b.layer0; p.k_blocks = cfg->k_blocks; p.cap_blocks = cfg->cap_blocks;
   p.thetabar_mode = cfg->thetabar_mode; p.beta = cfg->beta;
-  const size_t sm_sel = size_t(cfg->n_cap) * 4;
+  const size_t sm_sel = size_t(cfg->n_cap) * 8;        // scores and keys
   const bool fused = b.n_layers == 1 && cfg->n_kv_heads <= 8 && cfg->cap_blocks > 0;
   auto kern = fused ? select_kernel<true> : select_kernel<false>;
   if (sm_sel > 40 * 1024 &&
