@@ -292,19 +292,12 @@ class RetrievalState:
              advance=True, overlap_append=False):
         """bias -> probe -> score -> cut-off/select -> attention -> append for every unit.
 
-        overlap_append: enqueue the append on a second stream, concurrent with the other five
-        stages (it reads only the step's own K / V and writes pages and table rows that the other
-        stages of the same step do not read); the streams are joined before the step returns."""
+        overlap_append: enqueue the append on a second stream, concurrent with the attention (it
+        reads only the step's own K / V and writes pages and table rows that the attention of the
+        same step does not read); the streams are joined before the step returns."""
         cfg, b = self.cfg, self.batch
         nt = n_tokens if n_tokens is not None else q.shape[-3]
         main = torch.cuda.current_stream()
-        if overlap_append:
-            if getattr(self, "_side", None) is None:
-                self._side = torch.cuda.Stream(device=self.device)
-            self._side.wait_stream(main)
-            with torch.cuda.stream(self._side):
-                append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
-                              self.repr_k, self.repr_inv_norm, self.status)
         if update_probe:
             if fused:
                 bias_probe(cfg, b, q, nt, self.stats_count, self.stats_mean, self.stats_m2, self.phi_l1,
@@ -322,6 +315,13 @@ class RetrievalState:
                          self.scores, self.theta, self.status)
             select_cutoff(cfg, b, self.scores, self.theta, self.n_cand, self.budget_state, self.sel_idx,
                           self.sel_count, self.budget_real, self.status)
+        if overlap_append:
+            if getattr(self, "_side", None) is None:
+                self._side = torch.cuda.Stream(device=self.device)
+            self._side.wait_stream(main)
+            with torch.cuda.stream(self._side):
+                append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
+                              self.repr_k, self.repr_inv_norm, self.status)
         retrieval_attention(cfg, b, q, k_win, v_win, nt, self.k_pages, self.v_pages, self.page_table,
                             self.pos0, self.sel_idx, self.sel_count, out, lse, self.status)
         if overlap_append:

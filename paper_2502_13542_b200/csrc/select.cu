@@ -26,7 +26,6 @@ namespace {
 
 constexpr int kChainThreads = 1024;
 constexpr int kSelThreads = 256;
-constexpr int kRestCap = 128;          // deeper layers whose mean densities are divided out in parallel
 
 struct ChainParams {
   const float* scores;
@@ -176,6 +175,72 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* t
   return base + inc - v;
 }
 
+// Eq. 11 for one head by the whole CTA (kSelThreads threads): the same quantities as warp_entropy,
+// partial sums per thread, then per warp, then over the warps in a fixed order.  Every thread
+// returns theta.  red: 3 * (kSelThreads / 32) floats of shared memory; contains a CTA barrier.
+__device__ __forceinline__ float block_entropy(const float* sc, int n, float beta, float* red) {
+  constexpr int NW = kSelThreads / 32;
+  if (n <= 0) return 0.f;                       // uniform over the CTA
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float m = -INFINITY;
+  for (int i = tid; i < n; i += kSelThreads) m = fmaxf(m, beta * sc[i]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < NW; ++w) m = fmaxf(m, red[w]);
+  float z = 0.f, ex = 0.f;
+  for (int i = tid; i < n; i += kSelThreads) {
+    const float x = beta * sc[i] - m;
+    const float e = expf(x);
+    z += e;
+    ex = fmaf(e, x, ex);
+  }
+  z = warp_sum(z);
+  ex = warp_sum(ex);
+  if (lane == 0) { red[NW + warp] = z; red[2 * NW + warp] = ex; }
+  __syncthreads();
+  z = 0.f; ex = 0.f;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) { z += red[NW + w]; ex += red[2 * NW + w]; }
+  return fmaxf(logf(z) - ex / z, 0.f);
+}
+
+// Up to kSelThreads candidates, one per thread: the number of candidates that come before this
+// thread's in the order of the selection (higher key first, equal keys by lower index).  Every
+// thread counts the keys greater than its own against all of them, four per shared-memory load;
+// candidates with equal keys get equal counts, which a histogram of the counts detects, and only
+// those threads then add the number of their equals with a lower index.  Contains CTA barriers;
+// threads past n return n.
+__device__ __forceinline__ int rank_of_candidate(const float* sc, int n, uint32_t* key_s, int* rank_s, int* cnt_s) {
+  const int tid = threadIdx.x;
+  const uint32_t mine = tid < n ? score_key(sc[tid]) : 0u;
+  key_s[tid] = mine;                            // the padding is the lowest key: never greater
+  cnt_s[tid] = 0;
+  __syncthreads();
+  const uint4* k4 = reinterpret_cast<const uint4*>(key_s);
+  const int n4 = (n + 3) >> 2;
+  int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+  auto count4 = [&](const uint4& v) { r0 += v.x > mine; r1 += v.y > mine; r2 += v.z > mine; r3 += v.w > mine; };
+  int q = 0;
+  for (; q + 4 <= n4; q += 4) {                 // four loads in flight before the first compare
+    const uint4 a = k4[q], b = k4[q + 1], c = k4[q + 2], d = k4[q + 3];
+    count4(a); count4(b); count4(c); count4(d);
+  }
+  for (; q < n4; ++q) count4(k4[q]);
+  int r = (r0 + r1) + (r2 + r3);
+  if (tid >= n) r = n;
+  rank_s[tid] = r;
+  if (tid < n) atomicAdd(&cnt_s[r], 1);
+  __syncthreads();
+  if (tid < n && cnt_s[r] > 1) {
+    int before = 0;
+    for (int j = 0; j < tid; ++j) before += rank_s[j] == r;
+    r += before;
+  }
+  return r;
+}
+
 // kFused: the call holds one layer; the grid is launched as clusters of n_kv_heads CTAs (one
 // sequence each) and the cut-off chain of that layer is evaluated here (ch), else sel_count is
 // an input written by cutoff_chain_kernel.
@@ -187,15 +252,15 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
   extern __shared__ uint32_t sel_smem[];       // the head's scores [n_cap] (fp32), then their keys [n_cap]
   float* sc = reinterpret_cast<float*>(sel_smem);
   uint32_t* keys = sel_smem + n_cap;
-  __shared__ unsigned long long key64[kSelThreads];
+  __shared__ __align__(16) uint32_t key_s[kSelThreads];
+  __shared__ int rank_s[kSelThreads];
   __shared__ int hist[256];
   __shared__ int warp_tot[kSelThreads / 32];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_need;
-  __shared__ float sh_theta;                   // this head's density (read by the cluster peers)
+  __shared__ float sh_thetas[8];               // the densities of the cluster's heads (written by their CTAs)
+  __shared__ float red_f[3 * (kSelThreads / 32)];
   __shared__ int sh_count;
-  __shared__ double rest_q[kRestCap];          // mean density of each deeper layer with a history
-  __shared__ unsigned char rest_has[kRestCap];
   __shared__ double sh_brem, sh_rest;
   __shared__ int sh_no_hist;
   const int g = blockIdx.x, unit = blockIdx.y, tid = threadIdx.x;
@@ -205,6 +270,8 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
   const float* s = scores + (size_t(unit) * n_kv_heads + g) * n_cap;
   // the scores are fetched once, by all threads at a time; density and selection read them from here
   for (int i = tid; i < n; i += kSelThreads) sc[i] = s[i];
+  const bool small = n <= kSelThreads;      // one candidate per thread: ranked by counting
+  int rank = 0;
   int c;
   if constexpr (kFused) {
     cg::cluster_group cluster = cg::this_cluster();
@@ -212,54 +279,46 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
     const int layer = ch.layer0;
     double* st = ch.state + size_t(seq) * (1 + 2 * ch.L);
     // The old state is read by every CTA before the cluster barrier, written by CTA 0 after it.
-    // The deeper layers' mean densities are divided out by one thread per layer; thread 32 then
-    // adds them in layer order (the order of the serial loop, so the sum has the same bits) while
-    // warp 0 takes this head's density.
-    const int deeper = ch.L - (layer + 1);
-    const bool spread = deeper <= kRestCap;
-    if (spread && tid >= 32) {
-      for (int t = tid - 32; t < deeper; t += kSelThreads - 32) {
-        const int j = layer + 1 + t;
+    // Warp 1 adds up the mean densities of the deeper layers that have a history (a lane per
+    // layer, then a butterfly over the lanes) while the scores arrive.
+    if (tid >= 32 && tid < 64) {
+      const int lane = tid - 32;
+      double part = 0.0;
+      int none = 0;
+      for (int j = layer + 1 + lane; j < ch.L; j += 32) {
         const double cnt = st[1 + ch.L + j];
-        rest_has[t] = cnt > 0.0;
-        rest_q[t] = cnt > 0.0 ? st[1 + j] / cnt : 0.0;
+        if (cnt > 0.0) part += st[1 + j] / cnt; else ++none;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        part += __shfl_xor_sync(0xffffffffu, part, o);
+        none += __shfl_xor_sync(0xffffffffu, none, o);
+      }
+      if (lane == 0) {
+        sh_brem = layer == 0 ? double(ch.L) * double(ch.k_blocks) : st[0];
+        sh_rest = part;
+        sh_no_hist = none;
       }
     }
     __syncthreads();
-    if (tid == 32) {
-      double rest_hist = 0.0;
-      int no_hist = 0;
-      if (spread) {
-        for (int t = 0; t < deeper; ++t) {
-          if (rest_has[t]) rest_hist += rest_q[t]; else ++no_hist;
-        }
-      } else {
-        for (int j = layer + 1; j < ch.L; ++j) {
-          const double cnt = st[1 + ch.L + j];
-          if (cnt > 0.0) rest_hist += st[1 + j] / cnt; else ++no_hist;
-        }
-      }
-      sh_brem = layer == 0 ? double(ch.L) * double(ch.k_blocks) : st[0];
-      sh_rest = rest_hist;
-      sh_no_hist = no_hist;
-    }
-    if (tid < 32) {
+    // this head's density, by the whole CTA; handed to every CTA of the cluster (one per KV head)
+    // by remote stores ahead of the cluster barrier, so that nobody reads a peer's memory after it
+    // and no CTA has to wait for its peers before it leaves
+    {
       const size_t uh = size_t(unit) * n_kv_heads + g;
-      float th;
-      if (ch.theta_in) {
-        th = ch.theta_in[uh];
-      } else {
-        th = warp_entropy(sc, n, ch.beta);
-        if (tid == 0 && ch.theta_out) ch.theta_out[uh] = th;
-      }
-      if (tid == 0) sh_theta = th;
+      const float th = ch.theta_in ? ch.theta_in[uh] : block_entropy(sc, n, ch.beta, red_f);
+      if (tid == 0 && !ch.theta_in && ch.theta_out) ch.theta_out[uh] = th;
+      if (tid < n_kv_heads) cluster.map_shared_rank(sh_thetas, unsigned(tid))[g] = th;
     }
-    cluster.sync();
+    // arrive, rank this thread's candidate while the barrier completes (the ranks do not depend on
+    // the count), then wait
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    if (small) rank = rank_of_candidate(sc, n, key_s, rank_s, hist);
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
     if (tid == 0) {
-      float th_h[8];                             // all peers' values first: independent remote loads
+      float th_h[8];
 #pragma unroll
-      for (int h2 = 0; h2 < 8; ++h2)
-        th_h[h2] = h2 < n_kv_heads ? *cluster.map_shared_rank(&sh_theta, unsigned(h2)) : 0.f;
+      for (int h2 = 0; h2 < 8; ++h2) th_h[h2] = h2 < n_kv_heads ? sh_thetas[h2] : 0.f;
       double sum = 0.0;
 #pragma unroll
       for (int h2 = 0; h2 < 8; ++h2) sum += double(th_h[h2]);
@@ -289,6 +348,7 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
     __syncthreads();
     c = sh_count;
   } else {
+    if (small) rank = rank_of_candidate(sc, n, key_s, rank_s, hist);
     c = sel_count[unit];
     if (c < 0 || c > min(cap_blocks, n)) {
       if (tid == 0) set_status(status, ACTQKV_DEV_BAD_SELECTION);
@@ -299,17 +359,8 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
   for (int i = c + tid; i < cap_blocks; i += kSelThreads) out[i] = -1;
   if (c >= n) {
     for (int i = tid; i < min(n, c); i += kSelThreads) out[i] = i;
-  } else if (c > 0 && n <= kSelThreads) {
-    // One candidate per thread: its rank is the number of candidates that come before it in the
-    // order (higher key first, equal keys by lower index), counted against all of them; the c
-    // first are taken and compacted in ascending index order.
-    const uint32_t k = tid < n ? score_key(sc[tid]) : 0u;
-    key64[tid] = tid < n ? ((static_cast<unsigned long long>(k) << 32) | uint32_t(~uint32_t(tid))) : 0ull;
-    __syncthreads();
-    const unsigned long long mine = key64[tid];
-    int rank = 0;
-#pragma unroll 4
-    for (int j = 0; j < n; ++j) rank += key64[j] > mine;
+  } else if (c > 0 && small) {
+    // the c first of the order are taken and compacted in ascending index order
     const int take = tid < n && rank < c;
     int tot;
     const int pos = block_exclusive_scan(take, warp_tot, &tot);
@@ -389,7 +440,6 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
       }
     }
   }
-  if constexpr (kFused) cg::this_cluster().sync();   // peers may still be reading sh_theta
 }
 
 int launch_cutoff(const actqkv_config* cfg, const Batch& b, const float* scores, const float* theta_in,
