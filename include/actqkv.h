@@ -32,6 +32,16 @@
  *    representative-key table are caller-owned buffers updated in place).
  *  - Every call only ENQUEUES work on `stream` (a cudaStream_t passed as void*;
  *    NULL = the legacy default stream) and never synchronises.
+ *  - Stream order is kept for every result, but kernels of consecutive calls on
+ *    one stream may be RESIDENT together (programmatic dependent launch): the
+ *    kernels of steps 1-4 let the next kernel of the stream start at once, and a
+ *    kernel of this library that starts early reads, before it has waited for
+ *    its predecessor, only buffers that steps 1-5 never write: the step's Q / K /
+ *    V, pos0, page_table, the cache pages and table rows of tokens before pos0.
+ *    It waits for its predecessor before it reads anything else and before it
+ *    writes.  actqkv_append_window, which writes those buffers, runs strictly
+ *    after its predecessor and before its successor in the stream, and so does
+ *    a caller's own kernel between two calls unless it opts into the mechanism.
  *  - Return value: ACTQKV_OK (0) or a negative actqkv_status for problems the
  *    host can see (null / misaligned pointer, unsupported shape).  Nothing is
  *    enqueued when a negative code is returned.

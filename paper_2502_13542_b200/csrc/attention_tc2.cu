@@ -336,6 +336,14 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       issued = tiles_a + w + 1;
     }
     if (ok) {
+      // the page-table entries of every candidate block start their way into L2 while this warp
+      // sits in the wait: the look-ups of the selected blocks that follow it then find them there
+      if (!is_v) {
+        const char* pt0 = reinterpret_cast<const char*>(ks.pt + p.n_init / 16);
+        const int lines = min(ks.max_pages - p.n_init / 16, ks.n_cand * ks.gpb) / 32;     // 32 entries per 128 bytes
+        for (int l = lane; l < lines; l += 32)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(pt0 + size_t(l) * 128));
+      }
       const int n_tiles = total_after_wait(report && lane == 0);
       if (!is_v && lane == 0) mbar_arrive(bar_sel);      // the converter warps poll this instead of blocking
       paged_tiles(n1, n_tiles - n1, [&](int gi) { return page_b(ks, gi, p.a.status, report); });

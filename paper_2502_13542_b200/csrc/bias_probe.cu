@@ -198,30 +198,34 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
     cluster.sync();
     // ---- 2. merge the row splits, then the running statistics (Eq. 8 over all windows so far)
     if (tid < D) {
+      // every remote load is issued before the first use (a slot past S re-reads slot 0 and is
+      // dropped): loads under a condition would go out one at a time, a cluster round trip each
       float pn[kMaxCluster], pm[kMaxCluster], pm2[kMaxCluster];
 #pragma unroll
       for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-        pn[s2] = 0.f; pm[s2] = 0.f; pm2[s2] = 0.f;
-        if (s2 < S) {
-          const unsigned rk = unsigned(s2 + S * (cy > 1 ? hy : 0));
-          pn[s2] = cluster.map_shared_rank(scal, rk)[1];
-          pm[s2] = cluster.map_shared_rank(st_mean, rk)[tid];
-          pm2[s2] = cluster.map_shared_rank(st_m2, rk)[tid];
-        }
+        const unsigned rk = unsigned((s2 < S ? s2 : 0) + S * (cy > 1 ? hy : 0));
+        pn[s2] = cluster.map_shared_rank(scal, rk)[1];
+        pm[s2] = cluster.map_shared_rank(st_mean, rk)[tid];
+        pm2[s2] = cluster.map_shared_rank(st_m2, rk)[tid];
       }
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2)
+        if (s2 >= S) { pn[s2] = 0.f; pm[s2] = 0.f; pm2[s2] = 0.f; }
       double n = 0.0, mean = 0.0, m2 = 0.0;
 #pragma unroll
       for (int s2 = 0; s2 < kMaxCluster; ++s2) {
         const double nb = double(pn[s2]);
         if (nb == 0.0) continue;
-        const double nn = n + nb, delta = double(pm[s2]) - mean, w = nb / nn;
+        // the weights are ratios of token counts, the same in every thread: an fp32 division (a
+        // double one is some thirty dependent instructions, five of them in a row on this path)
+        const double nn = n + nb, delta = double(pm[s2]) - mean, w = double(float(nb) / float(nn));
         mean += delta * w;
         m2 += double(pm2[s2]) + delta * delta * (n * w);
         n = nn;
       }
       if (running) {
         const double na = double(run_count), mean_a = double(run_mean), m2_a = double(run_m2);
-        const double nn = na + n, delta = mean - mean_a, w = n / nn;
+        const double nn = na + n, delta = mean - mean_a, w = double(float(n) / float(nn));
         mean = mean_a + delta * w;
         m2 = m2_a + m2 + delta * delta * (na * w);
         n = nn;
@@ -231,9 +235,9 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
           if (tid == 0) p.stats_count[uh] = run_count + W;
         }
       }
-      const double var = n > 1.0 ? m2 / (n - 1.0) : 0.0;
+      const float var = n > 1.0 ? float(m2) / float(n - 1.0) : 0.f;      // sigma^2 and its inverse are fp32 results
       mean_s[tid] = float(mean);
-      ivar_s[tid] = float(1.0 / fmax(var, double(p.var_eps)));
+      ivar_s[tid] = 1.f / fmaxf(var, p.var_eps);
     }
     __syncthreads();
     // ---- 3. phi and its L1 norm a_j per token (the VPR lanes of a row add up by shuffles) and, with
@@ -311,15 +315,18 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
   if (sp == 0 && tid < D) {
     float tot[kMaxCluster], uu[kMaxCluster], qq[kMaxCluster];
     const int n_cta = S * cy;
+    const unsigned self = cluster.block_rank();
 #pragma unroll
-    for (int rk = 0; rk < kMaxCluster; ++rk) {
-      tot[rk] = 0.f; uu[rk] = 0.f; qq[rk] = 0.f;
-      if (rk < n_cta && (hy == 0 || rk / S == hy)) {
-        tot[rk] = cluster.map_shared_rank(scal, unsigned(rk))[0];
-        uu[rk] = cluster.map_shared_rank(u_s, unsigned(rk))[tid];
-        qq[rk] = cluster.map_shared_rank(qsum_s, unsigned(rk))[tid];
-      }
+    for (int rk = 0; rk < kMaxCluster; ++rk) {       // all loads first (see step 2); unused slots read this CTA
+      const bool used = rk < n_cta && (hy == 0 || rk / S == hy);
+      const unsigned src = used ? unsigned(rk) : self;
+      tot[rk] = cluster.map_shared_rank(scal, src)[0];
+      uu[rk] = cluster.map_shared_rank(u_s, src)[tid];
+      qq[rk] = cluster.map_shared_rank(qsum_s, src)[tid];
     }
+#pragma unroll
+    for (int rk = 0; rk < kMaxCluster; ++rk)
+      if (!(rk < n_cta && (hy == 0 || rk / S == hy))) { tot[rk] = 0.f; uu[rk] = 0.f; qq[rk] = 0.f; }
     auto head_probe = [&](int y) {
       float t = 0.f, u2 = 0.f, q2 = 0.f;
 #pragma unroll
