@@ -247,6 +247,7 @@ def run_ours(args):
                          "c": int(st0.sel_count.item())}
 
     side = torch.cuda.Stream(device=device)
+    ev_fork, ev_join = torch.cuda.Event(), torch.cuda.Event()
 
     def one_step(i, events=None, overlap=True):
         """One window through the six stages.  In the timed loop the append runs on a second stream,
@@ -258,8 +259,9 @@ def run_ours(args):
         st = states[i % n_copies]
         q, k, v, out = inputs[i % n_copies]
         b = st.batch
-        append = lambda: B.append_window(cfg, b, k, v, spec.window, st.pos0, st.k_pages, st.v_pages,
-                                         st.page_table, st.repr_k, st.repr_inv_norm, st.status)
+        append = lambda stream=None: B.append_window(cfg, b, k, v, spec.window, st.pos0, st.k_pages, st.v_pages,
+                                                     st.page_table, st.repr_k, st.repr_inv_norm, st.status,
+                                                     stream=stream)
         calls = (
             ("bias_probe", lambda: B.bias_probe(cfg, b, q, spec.window, st.stats_count, st.stats_mean, st.stats_m2,
                                                 st.phi_l1, None, st.probe_qh, st.probe_kv, st.status)),
@@ -281,13 +283,25 @@ def run_ours(args):
                 fn()
             return
         main = torch.cuda.current_stream()
+
+        def fork_append():
+            ev_fork.record(main)
+            side.wait_event(ev_fork)
+            append(side)
+            ev_join.record(side)
+
+        # Replayed from a graph the append starts with the attention, once the selection is done
+        # (earlier it competes with the short kernels the attention waits for); with plain
+        # launches an event recorded between two kernels of the chain would cost the second one
+        # its early start, so the fork sits in front of the step.
+        late = torch.cuda.is_current_stream_capturing()
+        if not late:
+            fork_append()
         for name, fn in calls:
-            if name == "attention":        # the append starts with the attention, once the selection is done
-                side.wait_stream(main)
-                with torch.cuda.stream(side):
-                    append()
+            if late and name == "attention":
+                fork_append()
             fn()
-        main.wait_stream(side)
+        main.wait_event(ev_join)
 
     launches_per_step = 5   # bias_probe, score, cut-off + select, attention, append
 

@@ -99,7 +99,17 @@ def _ptr(t):
     return t.data_ptr()
 
 
-def _stream():
+_raw_current_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream(stream=None):
+    """cudaStream_t of `stream`, or of the current stream of the current device.  (Building a
+    torch Stream object just to read its handle costs several microseconds per call, a third of
+    what it takes to enqueue one of these kernels.)"""
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_current_stream is not None:
+        return _raw_current_stream(torch.cuda.current_device())
     return torch.cuda.current_stream().cuda_stream
 
 
@@ -129,51 +139,51 @@ def n_candidates(cfg: Config, p0: int) -> int:
 
 
 def activation_bias(cfg, batch, q, n_tokens, stats_count, stats_mean, stats_m2, phi_l1,
-                    phi_full=None, status=None):
+                    phi_full=None, status=None, stream=None):
     _check(_lib.actqkv_activation_bias(C.byref(cfg), _b(batch), _ptr(q), n_tokens, _ptr(stats_count),
                                        _ptr(stats_mean), _ptr(stats_m2), _ptr(phi_l1), _ptr(phi_full),
-                                       _ptr(status), _stream()))
+                                       _ptr(status), _stream(stream)))
 
 
-def probe_query(cfg, batch, q, n_tokens, phi_l1, probe_qh, probe_kv, status=None):
+def probe_query(cfg, batch, q, n_tokens, phi_l1, probe_qh, probe_kv, status=None, stream=None):
     _check(_lib.actqkv_probe_query(C.byref(cfg), _b(batch), _ptr(q), n_tokens, _ptr(phi_l1),
-                                   _ptr(probe_qh), _ptr(probe_kv), _ptr(status), _stream()))
+                                   _ptr(probe_qh), _ptr(probe_kv), _ptr(status), _stream(stream)))
 
 
 def bias_probe(cfg, batch, q, n_tokens, stats_count, stats_mean, stats_m2, phi_l1, phi_full,
-               probe_qh, probe_kv, status=None):
+               probe_qh, probe_kv, status=None, stream=None):
     _check(_lib.actqkv_bias_probe(C.byref(cfg), _b(batch), _ptr(q), n_tokens, _ptr(stats_count),
                                   _ptr(stats_mean), _ptr(stats_m2), _ptr(phi_l1), _ptr(phi_full),
-                                  _ptr(probe_qh), _ptr(probe_kv), _ptr(status), _stream()))
+                                  _ptr(probe_qh), _ptr(probe_kv), _ptr(status), _stream(stream)))
 
 
-def score_blocks(cfg, batch, probe_kv, repr_k, repr_inv_norm, n_cand, scores, theta, status=None):
+def score_blocks(cfg, batch, probe_kv, repr_k, repr_inv_norm, n_cand, scores, theta, status=None, stream=None):
     _check(_lib.actqkv_score_blocks(C.byref(cfg), _b(batch), _ptr(probe_kv), _ptr(repr_k),
                                     _ptr(repr_inv_norm), _ptr(n_cand), _ptr(scores), _ptr(theta),
-                                    _ptr(status), _stream()))
+                                    _ptr(status), _stream(stream)))
 
 
 def select_cutoff(cfg, batch, scores, theta, n_cand, budget_state, sel_idx, sel_count,
-                  budget_real=None, status=None):
+                  budget_real=None, status=None, stream=None):
     _check(_lib.actqkv_select_cutoff(C.byref(cfg), _b(batch), _ptr(scores), _ptr(theta), _ptr(n_cand),
                                      _ptr(budget_state), _ptr(sel_idx), _ptr(sel_count),
-                                     _ptr(budget_real), _ptr(status), _stream()))
+                                     _ptr(budget_real), _ptr(status), _stream(stream)))
 
 
 def score_select(cfg, batch, probe_kv, repr_k, repr_inv_norm, n_cand, budget_state, scores, theta,
-                 sel_idx, sel_count, budget_real=None, status=None):
+                 sel_idx, sel_count, budget_real=None, status=None, stream=None):
     _check(_lib.actqkv_score_select(C.byref(cfg), _b(batch), _ptr(probe_kv), _ptr(repr_k),
                                     _ptr(repr_inv_norm), _ptr(n_cand), _ptr(budget_state), _ptr(scores),
                                     _ptr(theta), _ptr(sel_idx), _ptr(sel_count), _ptr(budget_real),
-                                    _ptr(status), _stream()))
+                                    _ptr(status), _stream(stream)))
 
 
 def retrieval_attention(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages, page_table, pos0,
-                        sel_idx, sel_count, out, lse=None, status=None):
+                        sel_idx, sel_count, out, lse=None, status=None, stream=None):
     _check(_lib.actqkv_retrieval_attention(C.byref(cfg), _b(batch), _ptr(q), _ptr(k_win), _ptr(v_win),
                                            n_tokens, _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
                                            _ptr(pos0), _ptr(sel_idx), _ptr(sel_count), _ptr(out),
-                                           _ptr(lse), _ptr(status), _stream()))
+                                           _ptr(lse), _ptr(status), _stream(stream)))
 
 
 def decode_splits(cfg, batch) -> int:
@@ -185,32 +195,32 @@ def decode_workspace_bytes(cfg, batch, n_tokens, n_splits=0) -> int:
 
 
 def decode_attention(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages, page_table, pos0,
-                     sel_idx, sel_count, out, lse=None, n_splits=0, workspace=None, status=None):
+                     sel_idx, sel_count, out, lse=None, n_splits=0, workspace=None, status=None, stream=None):
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(_lib.actqkv_decode_attention(C.byref(cfg), _b(batch), _ptr(q), _ptr(k_win), _ptr(v_win), n_tokens,
                                         _ptr(k_pages), _ptr(v_pages), _ptr(page_table), _ptr(pos0),
                                         _ptr(sel_idx), _ptr(sel_count), _ptr(out), _ptr(lse), n_splits,
-                                        _ptr(workspace), ws_bytes, _ptr(status), _stream()))
+                                        _ptr(workspace), ws_bytes, _ptr(status), _stream(stream)))
 
 
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
 def decode_attention_static(cfg, batch, q, k_win, v_win, n_tokens, k_pages, v_pages, page_table, pos0,
-                            sel_idx, sel_count, out, lse=None, n_splits=0, status=None):
+                            sel_idx, sel_count, out, lse=None, n_splits=0, status=None, stream=None):
     """The split decode attention with the library's own fixed scratch array: no workspace
     argument and no allocation.  Calls that may overlap on one GPU must not both use it."""
     _check(_lib.actqkv_decode_attention_static(C.byref(cfg), _b(batch), _ptr(q), _ptr(k_win), _ptr(v_win),
                                                n_tokens, _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
                                                _ptr(pos0), _ptr(sel_idx), _ptr(sel_count), _ptr(out), _ptr(lse),
-                                               n_splits, _ptr(status), _stream()))
+                                               n_splits, _ptr(status), _stream(stream)))
 
 
 def append_window(cfg, batch, k_win, v_win, n_tokens, pos0, k_pages, v_pages, page_table, repr_k,
-                  repr_inv_norm, status=None):
+                  repr_inv_norm, status=None, stream=None):
     _check(_lib.actqkv_append_window(C.byref(cfg), _b(batch), _ptr(k_win), _ptr(v_win), n_tokens,
                                      _ptr(pos0), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
-                                     _ptr(repr_k), _ptr(repr_inv_norm), _ptr(status), _stream()))
+                                     _ptr(repr_k), _ptr(repr_inv_norm), _ptr(status), _stream(stream)))
 
 
 # ----------------------------------------------------------------------------
@@ -292,12 +302,33 @@ class RetrievalState:
              advance=True, overlap_append=False):
         """bias -> probe -> score -> cut-off/select -> attention -> append for every unit.
 
-        overlap_append: enqueue the append on a second stream, concurrent with the attention (it
-        reads only the step's own K / V and writes pages and table rows that the attention of the
-        same step does not read); the streams are joined before the step returns."""
+        overlap_append: enqueue the append on a second stream, concurrent with the other stages (it
+        reads only the step's own K / V and writes pages and table rows that no other stage of the
+        same step reads); the streams are joined before the step returns."""
         cfg, b = self.cfg, self.batch
         nt = n_tokens if n_tokens is not None else q.shape[-3]
-        main = torch.cuda.current_stream()
+
+        def fork_append():
+            self._fork.record(main)
+            self._side.wait_event(self._fork)
+            append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
+                          self.repr_k, self.repr_inv_norm, self.status, stream=self._side)
+            self._join.record(self._side)
+
+        fork_late = False
+        if overlap_append:
+            if getattr(self, "_side", None) is None:
+                self._side = torch.cuda.Stream(device=self.device)
+            if getattr(self, "_fork", None) is None:
+                self._fork, self._join = torch.cuda.Event(), torch.cuda.Event()
+            main = torch.cuda.current_stream()
+            # Where the append forks off.  Inside a graph capture: after the selection, beside the
+            # attention (earlier it competes with the short kernels the attention waits for).  With
+            # plain launches an event recorded between two kernels of the chain would cost the
+            # second one its early start, so the fork sits in front of the whole step.
+            fork_late = torch.cuda.is_current_stream_capturing()
+            if not fork_late:
+                fork_append()
         if update_probe:
             if fused:
                 bias_probe(cfg, b, q, nt, self.stats_count, self.stats_mean, self.stats_m2, self.phi_l1,
@@ -315,17 +346,12 @@ class RetrievalState:
                          self.scores, self.theta, self.status)
             select_cutoff(cfg, b, self.scores, self.theta, self.n_cand, self.budget_state, self.sel_idx,
                           self.sel_count, self.budget_real, self.status)
-        if overlap_append:
-            if getattr(self, "_side", None) is None:
-                self._side = torch.cuda.Stream(device=self.device)
-            self._side.wait_stream(main)
-            with torch.cuda.stream(self._side):
-                append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
-                              self.repr_k, self.repr_inv_norm, self.status)
+        if fork_late:
+            fork_append()
         retrieval_attention(cfg, b, q, k_win, v_win, nt, self.k_pages, self.v_pages, self.page_table,
                             self.pos0, self.sel_idx, self.sel_count, out, lse, self.status)
         if overlap_append:
-            main.wait_stream(self._side)
+            main.wait_event(self._join)
         else:
             append_window(cfg, b, k_win, v_win, nt, self.pos0, self.k_pages, self.v_pages, self.page_table,
                           self.repr_k, self.repr_inv_norm, self.status)
