@@ -71,7 +71,15 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
   float* ivar_s = mean_s + D;                 // [D]
   float* red_s = ivar_s + D;                  // [32]
   float* a_s = red_s + 32;                    // [RP]
-  uint64_t* bar = reinterpret_cast<uint64_t*>(a_s + ((RP + 3) & ~3));
+  // records that OTHER CTAs of the cluster write into this one, ahead of a cluster barrier (so
+  // that nobody reads remote memory after a barrier and no CTA has to outlive its peers' reads)
+  float* rec_n = a_s + ((RP + 3) & ~3);       // [kMaxCluster] rows held by split s of this head
+  float* rec_mean = rec_n + kMaxCluster;      // [kMaxCluster][D] its mean
+  float* rec_m2 = rec_mean + kMaxCluster * D; // [kMaxCluster][D] its sum of squared deviations
+  float* prb_tot = rec_m2 + kMaxCluster * D;  // [kMaxCluster] sum_j a_j of cluster rank r (leaders only)
+  float* prb_u = prb_tot + kMaxCluster;       // [kMaxCluster][D] its sum_j a_j q_j
+  float* prb_q = prb_u + kMaxCluster * D;     // [kMaxCluster][D] its sum_j q_j
+  uint64_t* bar = reinterpret_cast<uint64_t*>(prb_q + kMaxCluster * D);
 
   const int sp = blockIdx.x, h = blockIdx.y, unit = blockIdx.z;
   const int hy = h % p.group;                 // head inside its KV group
@@ -195,22 +203,29 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
 #pragma unroll
   for (int e = 0; e < VN; ++e) acc[e] = 0.f;
   if (p.do_bias) {
+    // this CTA's record goes to every split of its head (itself included)
+    if (tid < D) {
+#pragma unroll
+      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
+        if (s2 < S) {
+          const unsigned rk = unsigned(s2 + S * (cy > 1 ? hy : 0));
+          cluster.map_shared_rank(rec_mean, rk)[sp * D + tid] = st_mean[tid];
+          cluster.map_shared_rank(rec_m2, rk)[sp * D + tid] = st_m2[tid];
+          if (tid == 0) cluster.map_shared_rank(rec_n, rk)[sp] = float(nr);
+        }
+      }
+    }
     cluster.sync();
     // ---- 2. merge the row splits, then the running statistics (Eq. 8 over all windows so far)
     if (tid < D) {
-      // every remote load is issued before the first use (a slot past S re-reads slot 0 and is
-      // dropped): loads under a condition would go out one at a time, a cluster round trip each
       float pn[kMaxCluster], pm[kMaxCluster], pm2[kMaxCluster];
 #pragma unroll
       for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-        const unsigned rk = unsigned((s2 < S ? s2 : 0) + S * (cy > 1 ? hy : 0));
-        pn[s2] = cluster.map_shared_rank(scal, rk)[1];
-        pm[s2] = cluster.map_shared_rank(st_mean, rk)[tid];
-        pm2[s2] = cluster.map_shared_rank(st_m2, rk)[tid];
+        const bool used = s2 < S;
+        pn[s2] = used ? rec_n[s2] : 0.f;
+        pm[s2] = used ? rec_mean[s2 * D + tid] : 0.f;
+        pm2[s2] = used ? rec_m2[s2 * D + tid] : 0.f;
       }
-#pragma unroll
-      for (int s2 = 0; s2 < kMaxCluster; ++s2)
-        if (s2 >= S) { pn[s2] = 0.f; pm[s2] = 0.f; pm2[s2] = 0.f; }
       double n = 0.0, mean = 0.0, m2 = 0.0;
 #pragma unroll
       for (int s2 = 0; s2 < kMaxCluster; ++s2) {
@@ -279,10 +294,7 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
     for (int r = tid; r < nr; r += kThreads) a_s[r] = p.phi_l1[uh * W + r0 + r];
     __syncthreads();
   }
-  if (!p.do_probe) {
-    if (p.do_bias) cluster.sync();      // peers may still be reading this CTA's record in step 2
-    return;
-  }
+  if (!p.do_probe) return;
 
   // ---- 4. this CTA's share of ||Phi||_1 and of sum_j a_j q_j
   {
@@ -303,10 +315,22 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
       }
     }
     column_reduce2(acc, zero, u_s, mean_s);      // mean_s is free by now: dummy destination
+    // this CTA's sums go to the leader of its head and to the leader of its KV group (rank 0)
+    const unsigned me = cluster.block_rank();
+    const unsigned head_leader = unsigned(S * (cy > 1 ? hy : 0));
     if (tid == 0) {
       float t = 0.f;
       for (int i = 0; i < kThreads / 32; ++i) t += red_s[i];
-      scal[0] = t;
+      cluster.map_shared_rank(prb_tot, head_leader)[me] = t;
+      if (head_leader != 0) cluster.map_shared_rank(prb_tot, 0)[me] = t;
+    }
+    if (tid < D) {
+      cluster.map_shared_rank(prb_u, head_leader)[me * D + tid] = u_s[tid];
+      cluster.map_shared_rank(prb_q, head_leader)[me * D + tid] = qsum_s[tid];
+      if (head_leader != 0) {
+        cluster.map_shared_rank(prb_u, 0)[me * D + tid] = u_s[tid];
+        cluster.map_shared_rank(prb_q, 0)[me * D + tid] = qsum_s[tid];
+      }
     }
   }
   cluster.sync();
@@ -315,18 +339,13 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
   if (sp == 0 && tid < D) {
     float tot[kMaxCluster], uu[kMaxCluster], qq[kMaxCluster];
     const int n_cta = S * cy;
-    const unsigned self = cluster.block_rank();
 #pragma unroll
-    for (int rk = 0; rk < kMaxCluster; ++rk) {       // all loads first (see step 2); unused slots read this CTA
+    for (int rk = 0; rk < kMaxCluster; ++rk) {
       const bool used = rk < n_cta && (hy == 0 || rk / S == hy);
-      const unsigned src = used ? unsigned(rk) : self;
-      tot[rk] = cluster.map_shared_rank(scal, src)[0];
-      uu[rk] = cluster.map_shared_rank(u_s, src)[tid];
-      qq[rk] = cluster.map_shared_rank(qsum_s, src)[tid];
+      tot[rk] = used ? prb_tot[rk] : 0.f;
+      uu[rk] = used ? prb_u[rk * D + tid] : 0.f;
+      qq[rk] = used ? prb_q[rk * D + tid] : 0.f;
     }
-#pragma unroll
-    for (int rk = 0; rk < kMaxCluster; ++rk)
-      if (!(rk < n_cta && (hy == 0 || rk / S == hy))) { tot[rk] = 0.f; uu[rk] = 0.f; qq[rk] = 0.f; }
     auto head_probe = [&](int y) {
       float t = 0.f, u2 = 0.f, q2 = 0.f;
 #pragma unroll
@@ -341,7 +360,6 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
       p.probe_kv[(size_t(unit) * p.n_kv_heads + h / p.group) * D + tid] = acc / float(p.group);
     }
   }
-  cluster.sync();      // peers keep their shared memory alive until the leaders have read it
 }
 
 // The N / 2 packed fp32 pairs of a 16-byte vector (element 2i in the low half of pair i).
@@ -808,7 +826,8 @@ int launch_d(const actqkv_config* cfg, const Batch& b, BiasProbeParams& p, cudaS
     if (!encode_q<T, D>(&tm_q, p, b.units(), p.box_rows)) return ACTQKV_ERR_LAUNCH;
     const size_t tile_bytes = (size_t(p.rows_alloc) * D * sizeof(T) + 127) & ~size_t(127);
     const size_t smem = tile_bytes + sizeof(float) * (size_t(2) * RL * D + 2 * NP * D + 6 * D + 4 + 32 +
-                                                       ((p.rows_per_cta + 3) & ~3)) + 16;
+                                                       ((p.rows_per_cta + 3) & ~3) + 2 * kMaxCluster +
+                                                       4 * kMaxCluster * D) + 16;
     if (smem > 220 * 1024) return ACTQKV_ERR_SHAPE;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
       return ACTQKV_ERR_LAUNCH;
