@@ -218,24 +218,19 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
     cluster.sync();
     // ---- 2. merge the row splits, then the running statistics (Eq. 8 over all windows so far)
     if (tid < D) {
-      float pn[kMaxCluster], pm[kMaxCluster], pm2[kMaxCluster];
-#pragma unroll
-      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-        const bool used = s2 < S;
-        pn[s2] = used ? rec_n[s2] : 0.f;
-        pm[s2] = used ? rec_mean[s2 * D + tid] : 0.f;
-        pm2[s2] = used ? rec_m2[s2 * D + tid] : 0.f;
-      }
+      // Rolled loops here and in step 5: these phases run once per launch, and straight-line code
+      // that is executed once costs its instruction fetch (the unrolled forms took twice as long
+      // inside a step as back to back with warm instructions).
       double n = 0.0, mean = 0.0, m2 = 0.0;
-#pragma unroll
-      for (int s2 = 0; s2 < kMaxCluster; ++s2) {
-        const double nb = double(pn[s2]);
+#pragma unroll 1
+      for (int s2 = 0; s2 < S; ++s2) {
+        const double nb = double(rec_n[s2]);
         if (nb == 0.0) continue;
         // the weights are ratios of token counts, the same in every thread: an fp32 division (a
         // double one is some thirty dependent instructions, five of them in a row on this path)
-        const double nn = n + nb, delta = double(pm[s2]) - mean, w = double(float(nb) / float(nn));
+        const double nn = n + nb, delta = double(rec_mean[s2 * D + tid]) - mean, w = double(float(nb) / float(nn));
         mean += delta * w;
-        m2 += double(pm2[s2]) + delta * delta * (n * w);
+        m2 += double(rec_m2[s2 * D + tid]) + delta * delta * (n * w);
         n = nn;
       }
       if (running) {
@@ -337,27 +332,24 @@ __global__ void __launch_bounds__(kThreads, 1) bias_probe_kernel(const __grid_co
   // ---- 5. Eq. 9 per query head, and the KV-head probe = mean over the G heads of the group.
   // The group leader repeats the per-head arithmetic in the same order, so both agree bitwise.
   if (sp == 0 && tid < D) {
-    float tot[kMaxCluster], uu[kMaxCluster], qq[kMaxCluster];
-    const int n_cta = S * cy;
-#pragma unroll
-    for (int rk = 0; rk < kMaxCluster; ++rk) {
-      const bool used = rk < n_cta && (hy == 0 || rk / S == hy);
-      tot[rk] = used ? prb_tot[rk] : 0.f;
-      uu[rk] = used ? prb_u[rk * D + tid] : 0.f;
-      qq[rk] = used ? prb_q[rk * D + tid] : 0.f;
-    }
-    auto head_probe = [&](int y) {
+    auto head_probe = [&](int y) {                 // ranks y * S .. y * S + S - 1 hold head y of the group
       float t = 0.f, u2 = 0.f, q2 = 0.f;
-#pragma unroll
-      for (int rk = 0; rk < kMaxCluster; ++rk)
-        if (rk >= y * S && rk < (y + 1) * S) { t += tot[rk]; u2 += uu[rk]; q2 += qq[rk]; }
+#pragma unroll 1
+      for (int rk = y * S; rk < (y + 1) * S; ++rk) { t += prb_tot[rk]; u2 += prb_u[rk * D + tid]; q2 += prb_q[rk * D + tid]; }
       return (t > 0.f && !p.mean_pool) ? u2 / t : q2 / float(W);      // all-zero bias: uniform weights
     };
-    p.probe_qh[hd + tid] = head_probe(cy > 1 ? hy : 0);
     if (hy == 0) {
-      float acc = 0.f;
-      for (int y = 0; y < p.group; ++y) acc += head_probe(y);
+      float acc = 0.f, own = 0.f;
+#pragma unroll 1
+      for (int y = 0; y < cy; ++y) {
+        const float pr = head_probe(y);
+        if (y == 0) own = pr;
+        acc += pr;
+      }
+      p.probe_qh[hd + tid] = own;
       p.probe_kv[(size_t(unit) * p.n_kv_heads + h / p.group) * D + tid] = acc / float(p.group);
+    } else {
+      p.probe_qh[hd + tid] = head_probe(hy);
     }
   }
 }
