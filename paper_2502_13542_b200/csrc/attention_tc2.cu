@@ -145,14 +145,18 @@ __device__ __forceinline__ int page_a(const PairKeys& ks, int gi, int32_t* statu
   return physical_page(ks, gi < ks.g_init ? int64_t(gi) : ks.local_page0 + (gi - ks.g_init), status, report);
 }
 // Part B, granule gi: the selected blocks in the order of sel_idx.
-__device__ __forceinline__ int page_b(const PairKeys& ks, int gi, int32_t* status, bool report) {
+// (blk = the entry of sel_idx that granule gi falls into, read by the caller)
+__device__ __forceinline__ int page_b_of_block(const PairKeys& ks, int gi, int blk, int32_t* status, bool report) {
   if (gi >= ks.g_b) return ks.page_oob;
-  const int blk = ks.sel[gi / ks.gpb];
   if (blk < 0 || blk >= ks.n_cand) {
     if (report) set_status(status, ACTQKV_DEV_BAD_SELECTION);
     return ks.page_oob;
   }
   return physical_page(ks, (int64_t(ks.n_init) + int64_t(blk) * ks.block) / 16 + gi % ks.gpb, status, report);
+}
+__device__ __forceinline__ int page_b(const PairKeys& ks, int gi, int32_t* status, bool report) {
+  if (gi >= ks.g_b) return ks.page_oob;
+  return page_b_of_block(ks, gi, ks.sel[gi / ks.gpb], status, report);
 }
 
 // ---------------------------------------------------------------- kernel
@@ -305,8 +309,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     // page_table, two dependent loads) are taken 32 granules = 4 tiles at a time, one granule per
     // lane, one chunk ahead of the tiles being issued, so that their latency is off the per-tile
     // path; the issuing lane fetches its page with a shuffle.
-    auto paged_tiles = [&](int j_base, int cnt, auto&& page_of) {
-      int page_cur = 0, page_next = page_of(lane);
+    auto paged_tiles = [&](int j_base, int cnt, auto&& page_of, int first_chunk) {
+      int page_cur = 0, page_next = first_chunk;
       for (int t = 0; t < cnt && ok; ++t) {
         if ((t & 3) == 0) page_cur = page_next;
         const int page = __shfl_sync(0xffffffffu, page_cur, (t & 3) * 8 + my_granule);
@@ -322,7 +326,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         if ((t & 3) == 0) page_next = page_of(((t >> 2) + 1) * 32 + lane);
       }
     };
-    paged_tiles(0, tiles_a, [&](int gi) { return page_a(ks, gi, p.a.status, report); });
+    paged_tiles(0, tiles_a, [&](int gi) { return page_a(ks, gi, p.a.status, report); }, page_a(ks, lane, p.a.status, report));
     for (int w = 0; w <= mt && ok; ++w) {
       uint32_t full = 0;
       const uint32_t sbase = claim(tiles_a + w, full);
@@ -344,9 +348,14 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int l = lane; l < lines; l += 32)
           asm volatile("prefetch.global.L2 [%0];" ::"l"(pt0 + size_t(l) * 128));
       }
+      // the first look-up into the selection goes out together with the load of the count
+      grid_dependency_wait();
+      const int e0 = lane / ks.gpb;
+      const int blk0 = e0 < p.cap_blocks ? ks.sel[e0] : -1;
       const int n_tiles = total_after_wait(report && lane == 0);
       if (!is_v && lane == 0) mbar_arrive(bar_sel);      // the converter warps poll this instead of blocking
-      paged_tiles(n1, n_tiles - n1, [&](int gi) { return page_b(ks, gi, p.a.status, report); });
+      paged_tiles(n1, n_tiles - n1, [&](int gi) { return page_b(ks, gi, p.a.status, report); },
+                  page_b_of_block(ks, lane, blk0, p.a.status, report));
     }
     // drain: what this CTA issued must have landed before it may leave on the abort path; its
     // copies complete on the leader's barriers, which only the leader can poll, so the peer waits
