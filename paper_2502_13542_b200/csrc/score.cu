@@ -223,14 +223,17 @@ score_kernel(const float* __restrict__ probe_kv, const T* __restrict__ repr_k,
   }
 }
 
-__global__ void __launch_bounds__(32)
+constexpr int kEntropyThreads = 256;
+
+__global__ void __launch_bounds__(kEntropyThreads)
 entropy_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_cand,
                float* __restrict__ theta, int n_kv_heads, int n_cap, int n_layers, float beta) {
+  __shared__ float red[3 * (kEntropyThreads / 32)];
   const int g = blockIdx.x, unit = blockIdx.y;
   grid_launch_dependents();
   grid_dependency_wait();            // the scores come from the stream's previous kernel
   const int n = min(n_cand[unit / n_layers], n_cap);
-  const float th = warp_entropy(scores + (size_t(unit) * n_kv_heads + g) * n_cap, n, beta);
+  const float th = block_entropy<kEntropyThreads>(scores + (size_t(unit) * n_kv_heads + g) * n_cap, n, beta, red);
   if (threadIdx.x == 0) theta[size_t(unit) * n_kv_heads + g] = th;
 }
 
@@ -289,7 +292,7 @@ int launch_entropy(const actqkv_config* cfg, const Batch& b, const float* scores
   prefer_max_shared(entropy_kernel);
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(cfg->n_kv_heads, b.units(), 1);
-  lc.blockDim = dim3(32, 1, 1);
+  lc.blockDim = dim3(kEntropyThreads, 1, 1);
   lc.stream = st;
   cudaLaunchAttribute attr[1];
   allow_early_launch(attr[0]);       // resident while the score kernel drains; waits for it before reading

@@ -59,16 +59,18 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
   grid_launch_dependents();
   grid_dependency_wait();            // scores / densities come from the stream's previous kernels
   const int n = min(p.n_cand[seq], p.n_cap);
-  for (int pair = warp; pair < p.Lb * p.n_kv_heads; pair += kChainThreads / 32) {
-    const size_t uh = size_t(seq) * p.Lb * p.n_kv_heads + pair;
-    float th;
-    if (p.theta_in) {
-      th = p.theta_in[uh];
-    } else {
-      th = warp_entropy(p.scores + uh * p.n_cap, n, p.beta);
-      if (lane == 0 && p.theta_out) p.theta_out[uh] = th;
+  if (p.theta_in) {                  // one load per thread, all in flight together
+    const float* src = p.theta_in + size_t(seq) * p.Lb * p.n_kv_heads;
+    for (int pair = threadIdx.x; pair < p.Lb * p.n_kv_heads; pair += kChainThreads) theta_h[pair] = src[pair];
+  } else {
+    for (int pair = warp; pair < p.Lb * p.n_kv_heads; pair += kChainThreads / 32) {
+      const size_t uh = size_t(seq) * p.Lb * p.n_kv_heads + pair;
+      const float th = warp_entropy(p.scores + uh * p.n_cap, n, p.beta);
+      if (lane == 0) {
+        if (p.theta_out) p.theta_out[uh] = th;
+        theta_h[pair] = th;
+      }
     }
-    if (lane == 0) theta_h[pair] = th;
   }
   __syncthreads();
 
@@ -100,12 +102,13 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
     suf_open[tid] = open;
   }
   __syncthreads();
-  if (tid == 0) {                    // suffix[j] = sum over layers >= j (additions only)
-    suf_known[p.L] = 0.0;
-    suf_open[p.L] = 0.0;
+  if (tid < 2) {                     // suffix[j] = sum over layers >= j (additions only, running sum in a register)
+    double* suf = tid == 0 ? suf_known : suf_open;
+    double run = 0.0;
+    suf[p.L] = 0.0;
     for (int j = p.L - 1; j >= 0; --j) {
-      suf_known[j] += suf_known[j + 1];
-      suf_open[j] += suf_open[j + 1];
+      run += suf[j];
+      suf[j] = run;
     }
   }
   __syncthreads();
@@ -121,17 +124,22 @@ __global__ void __launch_bounds__(kChainThreads) cutoff_chain_kernel(ChainParams
   // ---- serial: the budget walks the layers shallow -> deep
   if (tid == 0) {
     double b_rem = st[0];
+    const double lo_d = double(min(1, n)), hi_d = double(min(p.cap_blocks, n));
     for (int l = 0; l < p.Lb; ++l) {
       const int layer = p.layer0 + l;
       if (layer == 0) b_rem = double(p.L) * double(p.k_blocks);
       int c = 0;
       double real = 0.0;
       if (n > 0) {
+        // The count stays a double on the path from one layer's budget to the next (the clamp
+        // bounds are small integers, so clamping the double and converting gives the same count
+        // as converting and clamping; a NaN budget counts as 0 before the clamp, as a conversion
+        // to int would make it); the integer for the store is taken off that path.
         real = ratio[l] >= 0.0 ? ratio[l] * b_rem : b_rem / double(p.L - layer);
         const double fl = floor(real + 0.5);
-        c = fl > 2.0e9 ? 2000000000 : (fl < -2.0e9 ? -2000000000 : int(fl));
-        c = max(min(1, n), min(c, min(p.cap_blocks, n)));
-        b_rem -= double(c);
+        const double cd = fmax(lo_d, fmin(fl == fl ? fl : 0.0, hi_d));
+        b_rem -= cd;
+        c = int(cd);
       }
       const size_t unit = size_t(seq) * p.Lb + l;
       p.sel_count[unit] = c;
@@ -173,37 +181,6 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* t
   }
   *total = tot;
   return base + inc - v;
-}
-
-// Eq. 11 for one head by the whole CTA (kSelThreads threads): the same quantities as warp_entropy,
-// partial sums per thread, then per warp, then over the warps in a fixed order.  Every thread
-// returns theta.  red: 3 * (kSelThreads / 32) floats of shared memory; contains a CTA barrier.
-__device__ __forceinline__ float block_entropy(const float* sc, int n, float beta, float* red) {
-  constexpr int NW = kSelThreads / 32;
-  if (n <= 0) return 0.f;                       // uniform over the CTA
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float m = -INFINITY;
-  for (int i = tid; i < n; i += kSelThreads) m = fmaxf(m, beta * sc[i]);
-  m = warp_max(m);
-  if (lane == 0) red[warp] = m;
-  __syncthreads();
-#pragma unroll
-  for (int w = 0; w < NW; ++w) m = fmaxf(m, red[w]);
-  float z = 0.f, ex = 0.f;
-  for (int i = tid; i < n; i += kSelThreads) {
-    const float x = beta * sc[i] - m;
-    const float e = expf(x);
-    z += e;
-    ex = fmaf(e, x, ex);
-  }
-  z = warp_sum(z);
-  ex = warp_sum(ex);
-  if (lane == 0) { red[NW + warp] = z; red[2 * NW + warp] = ex; }
-  __syncthreads();
-  z = 0.f; ex = 0.f;
-#pragma unroll
-  for (int w = 0; w < NW; ++w) { z += red[NW + w]; ex += red[2 * NW + w]; }
-  return fmaxf(logf(z) - ex / z, 0.f);
 }
 
 // Up to kSelThreads candidates, one per thread: the number of candidates that come before this
@@ -306,7 +283,7 @@ select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ n_ca
     // and no CTA has to wait for its peers before it leaves
     {
       const size_t uh = size_t(unit) * n_kv_heads + g;
-      const float th = ch.theta_in ? ch.theta_in[uh] : block_entropy(sc, n, ch.beta, red_f);
+      const float th = ch.theta_in ? ch.theta_in[uh] : block_entropy<kSelThreads>(sc, n, ch.beta, red_f);
       if (tid == 0 && !ch.theta_in && ch.theta_out) ch.theta_out[uh] = th;
       if (tid < n_kv_heads) cluster.map_shared_rank(sh_thetas, unsigned(tid))[g] = th;
     }

@@ -24,11 +24,43 @@ __device__ __forceinline__ float warp_entropy(const float* __restrict__ s, int n
   return fmaxf(logf(z) - ex / z, 0.f);
 }
 
+// Eq. 11 for one head by a whole CTA of kCtaThreads threads: the same quantities as warp_entropy,
+// partial sums per thread, then per warp, then over the warps in a fixed order.  Every thread
+// returns theta.  red: 3 * (kCtaThreads / 32) floats of shared memory; contains a CTA barrier.
+template <int kCtaThreads>
+__device__ __forceinline__ float block_entropy(const float* sc, int n, float beta, float* red) {
+  constexpr int NW = kCtaThreads / 32;
+  if (n <= 0) return 0.f;                       // uniform over the CTA
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float m = -INFINITY;
+  for (int i = tid; i < n; i += kCtaThreads) m = fmaxf(m, beta * sc[i]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < NW; ++w) m = fmaxf(m, red[w]);
+  float z = 0.f, ex = 0.f;
+  for (int i = tid; i < n; i += kCtaThreads) {
+    const float x = beta * sc[i] - m;
+    const float e = expf(x);
+    z += e;
+    ex = fmaf(e, x, ex);
+  }
+  z = warp_sum(z);
+  ex = warp_sum(ex);
+  if (lane == 0) { red[NW + warp] = z; red[2 * NW + warp] = ex; }
+  __syncthreads();
+  z = 0.f; ex = 0.f;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) { z += red[NW + w]; ex += red[2 * NW + w]; }
+  return fmaxf(logf(z) - ex / z, 0.f);
+}
+
 int launch_scores(const actqkv_config* cfg, const Batch& b, const float* probe_kv, const void* repr_k,
                   const float* repr_inv_norm, const int32_t* n_cand, float* scores, int32_t* status,
                   cudaStream_t st);
 
-// Eq. 11 for every (unit, KV head), one warp each.
+// Eq. 11 for every (unit, KV head), one CTA each.
 int launch_entropy(const actqkv_config* cfg, const Batch& b, const float* scores, const int32_t* n_cand,
                    float* theta, cudaStream_t st);
 
