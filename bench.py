@@ -227,7 +227,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
-    spec = wl.llama3_8b_layer()
+    spec = wl.llama3_8b_layer().replace(page_tokens=args.page_tokens)
     p0 = (spec.n_windows - 1) * spec.window
     n_copies = args.copies
     extras = world == 1 and not args.headline_only
@@ -562,7 +562,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "llama3_8b_layer_32k: last window (p0=32256) of a 32768-token prefill, "
-                               "Hq=32 Hkv=8 D=128 W=512 B=128 r=4 n_init=128 k=cap=32, bf16 16-token pages",
+                               f"Hq=32 Hkv=8 D=128 W=512 B=128 r=4 n_init=128 k=cap=32, bf16 {spec.page_tokens}-token pages",
                    "cold_l2": f"{n_copies} distinct layer-state copies rotated (inputs larger than L2)",
                    "selected_blocks": c_sel, "parallelism": f"independent layers x{world}", "streams": "append on a second stream beside the attention, joined every step",
                    "launch": "eager calls" if args.eager else f"one CUDA graph of the {args.steps} steps, replayed per repetition"},
@@ -991,6 +991,8 @@ def main():
                          "the others print one secondary measurement alone")
     ap.add_argument("--stack-layers", type=int, default=32, help="stack32 workload: layers batched per launch")
     ap.add_argument("--reps", type=int, default=20, help="repetitions of the timed K-step region (median reported)")
+    ap.add_argument("--page-tokens", type=int, default=16, choices=[16, 32, 64, 128],
+                    help="tokens per cache page of the layer32k workload (the headline workload has 16)")
     ap.add_argument("--eager", action="store_true",
                     help="enqueue the timed steps call by call from Python instead of replaying a CUDA graph of them")
     ap.add_argument("--headline-only", action="store_true",

@@ -246,7 +246,7 @@ int actqkv_score_select(const actqkv_config* cfg, const actqkv_batch* batch, con
  *   out          [U][n_tokens][Hq][D]   cfg->out_dtype out
  *   lse          [U][Hq][n_tokens]      fp32 out, may be NULL (natural-log sum of exp)
  * bf16, D = 128, 16-token pages: steps whose n_tokens is a multiple of 128 run on the tcgen05
- * prefill kernels (CTA pairs when G is even), steps of n_tokens <= 128 / G tokens on the tcgen05
+ * prefill kernels (CTA pairs when G is even; that kernel also takes pages of 32, 64 or 128 tokens), steps of n_tokens <= 128 / G tokens on the tcgen05
  * decode kernel (one CTA per KV head; see actqkv_decode_attention for the split form); every
  * other shape runs on the general fp32-accumulate kernel.
  * Preconditions of the tcgen05 kernels (the general kernel has none of them):

@@ -127,11 +127,15 @@ struct PairKeys {
   const int32_t* sel;
   const int32_t* pt;
   int g_init, g_a, g_b, gpb, n_cand, n_init, block, max_pages, n_phys_pages, page_base, page_oob;
-  int64_t local_page0;
+  int gpp;                   // 16-token granules per cache page (1, 2, 4 or 8)
+  int64_t local_page0;       // first granule of the local past, counted from token 0
 };
-// Row of the 4-D tensor map of logical page lp; page_oob (outside the tensor: TMA fills zeros) for
-// rejected table entries.
-__device__ __forceinline__ int physical_page(const PairKeys& ks, int64_t lp, int32_t* status, bool report) {
+// The key stream is addressed in granules of 16 tokens whatever the page size; a page of
+// 16 * gpp tokens holds gpp consecutive granules, and every part of the stream starts on a page.
+// Row of the 4-D tensor map of the page that holds granule lg (counted from token 0); page_oob
+// (outside the tensor: TMA fills zeros) for rejected table entries.
+__device__ __forceinline__ int physical_page(const PairKeys& ks, int64_t lg, int32_t* status, bool report) {
+  const int64_t lp = lg / ks.gpp;
   const int phys = lp < ks.max_pages ? ks.pt[lp] : -1;
   if (phys < 0 || phys >= ks.n_phys_pages) {
     if (report) set_status(status, ACTQKV_DEV_BAD_PAGE);
@@ -236,7 +240,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   PairKeys ks;
   ks.sel = p.a.sel_idx + (size_t(unit) * p.n_kv_heads + g) * p.cap_blocks;
   ks.pt = p.a.page_table + size_t(seq) * p.max_pages;
-  ks.gpb = p.block / 16;                                 // page granules per block
+  ks.gpb = p.block / 16;                                 // granules per block
+  ks.gpp = p.page_tokens / 16;
   ks.g_init = geo.init_len / 16;
   ks.g_a = ks.g_init + int((local_len + 15) / 16);       // the last local page may be partly filled
   ks.g_b = 0;
@@ -284,9 +289,17 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       tma2_load_3d(q_smem, &tm_q, leader_addr(bar_q), 0, h, unit * nt + mt * kBM);
       tma2_load_3d(q_smem + kSubTileBytes, &tm_q, leader_addr(bar_q), 64, h, unit * nt + mt * kBM);
     }
-    // lanes 0-7 issue one box each.  K: (channel half, granule 4 * rank + slot); V: granule = lane.
-    const int half = (lane >> 2) & 1, slot = lane & 3;
-    const int my_granule = is_v ? (lane & 7) : int(rank) * 4 + slot;
+    // One box per page (or per part of a page that belongs to this CTA's share of the tile) and,
+    // for K, per 64-channel half: with 16-token pages lanes 0-7 issue one box of 16 rows each
+    // (K: channel half, granule 4 * rank + slot; V: granule = lane), with larger pages fewer lanes
+    // issue taller boxes.  A box costs the copy engine about the same whatever its height.
+    const int box_g = min(ks.gpp, is_v ? 8 : 4);           // granules per box
+    const int n_box = is_v ? 8 / box_g : 2 * (4 / box_g);  // boxes of this CTA per tile
+    const int per_half = is_v ? n_box : n_box / 2;
+    const int half = lane / per_half, slot = lane % per_half;
+    const int my_granule = (is_v ? 0 : int(rank) * 4) + slot * box_g;          // first granule of the box, in the tile
+    const int tok_in_page = (my_granule % ks.gpp) * 16;
+    const uint32_t box_off = (is_v ? 0u : uint32_t(half) * kKSubBytes) + uint32_t(slot * box_g) * 2048u;
     const bool report = !is_v && leader;
     bool ok = true;
     int issued = 0;
@@ -317,9 +330,9 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         uint32_t full = 0;
         const uint32_t sbase = claim(j_base + t, full);
         if (!ok) break;
-        if (lane < 8) {
-          if (is_v) tma_load_4d(sbase + lane * 2048u, tm_pages, full, int(rank) * 64, 0, g, page);
-          else tma2_load_4d(sbase + half * kKSubBytes + slot * 2048u, tm_pages, full, half * 64, 0, g, page);
+        if (lane < n_box) {
+          if (is_v) tma_load_4d(sbase + box_off, tm_pages, full, int(rank) * 64, tok_in_page, g, page);
+          else tma2_load_4d(sbase + box_off, tm_pages, full, half * 64, tok_in_page, g, page);
         }
         issued = j_base + t + 1;
         // the next chunk of look-ups after the issue: its stall is behind the ring
@@ -343,8 +356,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       // the page-table entries of every candidate block start their way into L2 while this warp
       // sits in the wait: the look-ups of the selected blocks that follow it then find them there
       if (!is_v) {
-        const char* pt0 = reinterpret_cast<const char*>(ks.pt + p.n_init / 16);
-        const int lines = min(ks.max_pages - p.n_init / 16, ks.n_cand * ks.gpb) / 32;     // 32 entries per 128 bytes
+        const char* pt0 = reinterpret_cast<const char*>(ks.pt + p.n_init / p.page_tokens);
+        const int lines = min(ks.max_pages - p.n_init / p.page_tokens, ks.n_cand * ks.gpb / ks.gpp) / 32;     // 32 entries per 128 bytes
         for (int l = lane; l < lines; l += 32)
           asm volatile("prefetch.global.L2 [%0];" ::"l"(pt0 + size_t(l) * 128));
       }
@@ -679,8 +692,10 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 namespace actqkv {
 
 bool attention_tc2_supported(const actqkv_config* cfg, int n_tokens) {
-  const int group = cfg->n_q_heads / cfg->n_kv_heads;
-  return attention_tc_supported(cfg, n_tokens) && group % 2 == 0;
+  const int group = cfg->n_q_heads / cfg->n_kv_heads, P = cfg->page_tokens;
+  const bool page_ok = P == 16 || P == 32 || P == 64 || P == 128;
+  return cfg->dtype == ACTQKV_BF16 && cfg->head_dim == 128 && page_ok && n_tokens % kBM == 0 && cfg->block % P == 0 &&
+         cfg->n_init % P == 0 && cfg->n_local_prev % 16 == 0 && group % 2 == 0;
 }
 
 int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArgs& a, cudaStream_t st) {
@@ -701,17 +716,22 @@ int launch_attention_tc2(const actqkv_config* cfg, const Batch& b, const AttnArg
     if (!encode(&tm_vw, a.v_win, 3, dims, str, box_v)) return ACTQKV_ERR_LAUNCH;
   }
   {
-    const cuuint64_t dims[4] = {cuuint64_t(kD), 16, cuuint64_t(Hkv), cuuint64_t(b.n_layers) * cfg->n_phys_pages};
-    const cuuint64_t str[3] = {cuuint64_t(kD) * 2, cuuint64_t(kD) * 2 * 16, cuuint64_t(kD) * 2 * 16 * Hkv};
-    const cuuint32_t box[4] = {64, 16, 1, 1};
-    if (!encode(&tm_kp, a.k_pages, 4, dims, str, box)) return ACTQKV_ERR_LAUNCH;
-    if (!encode(&tm_vp, a.v_pages, 4, dims, str, box)) return ACTQKV_ERR_LAUNCH;
+    const cuuint64_t P = cuuint64_t(cfg->page_tokens);
+    const cuuint64_t dims[4] = {cuuint64_t(kD), P, cuuint64_t(Hkv), cuuint64_t(b.n_layers) * cfg->n_phys_pages};
+    const cuuint64_t str[3] = {cuuint64_t(kD) * 2, cuuint64_t(kD) * 2 * P, cuuint64_t(kD) * 2 * P * Hkv};
+    // a CTA holds 64 keys of a K tile and all 128 keys of its channel half of a V tile: a box is a
+    // whole page, or the part of a larger page that falls into that share
+    const cuuint32_t box_k[4] = {64, cuuint32_t(std::min(cfg->page_tokens, 64)), 1, 1};
+    const cuuint32_t box_v[4] = {64, cuuint32_t(std::min(cfg->page_tokens, 128)), 1, 1};
+    if (!encode(&tm_kp, a.k_pages, 4, dims, str, box_k)) return ACTQKV_ERR_LAUNCH;
+    if (!encode(&tm_vp, a.v_pages, 4, dims, str, box_v)) return ACTQKV_ERR_LAUNCH;
   }
   TcParams p;
   p.a = a;
   p.n_q_heads = Hq; p.n_kv_heads = Hkv; p.group = Hq / Hkv; p.block = cfg->block; p.n_init = cfg->n_init;
   p.n_local_prev = cfg->n_local_prev; p.cap_blocks = cfg->cap_blocks; p.max_pages = cfg->max_pages;
   p.n_phys_pages = cfg->n_phys_pages; p.n_layers = b.n_layers; p.out_bf16 = cfg->out_dtype == ACTQKV_BF16;
+  p.page_tokens = cfg->page_tokens;
   const float scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.f / sqrtf(float(kD));
   p.scale_log2 = scale * 1.4426950408889634f;
   static std::atomic<bool> opted_in[kMaxDevices];

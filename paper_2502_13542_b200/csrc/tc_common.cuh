@@ -20,6 +20,7 @@ struct TcParams {
   int n_q_heads, n_kv_heads, group, block, n_init, n_local_prev, cap_blocks;
   int max_pages, n_phys_pages, n_layers, out_bf16;
   float scale_log2;
+  int page_tokens = 16;        // tokens per cache page (the CTA-pair kernel takes 16, 32, 64 or 128)
 };
 
 // ---------------------------------------------------------------- PTX wrappers

@@ -109,3 +109,51 @@ def test_prefill_step_off_the_page_boundary(B):
                 pu.assert_attention(pu.to_numpy(o2), res["out"], f"unaligned p0 = {p0}, {nm}")
         st.set_positions([p0 + nt])
     assert int(st.status.item()) == 0
+
+
+@pytest.mark.parametrize("page_tokens", [32, 64, 128])
+def test_larger_cache_pages(B, page_tokens):
+    """Cache pages of 32, 64 and 128 tokens (the paged cache's page size is a deployment choice;
+    the other workloads use 16): every stage on the LLaMA shape, 8 windows of a 4096-token prefill,
+    shuffled page table, attention on the CTA-pair tensor-core kernel (one copy box per page, or
+    per part of a page inside a CTA's share of a tile) at windows {1, 7}."""
+    spec = wl.llama3_8b_layer().replace(context=4096, n_planted=3, page_tokens=page_tokens)
+    stats, o_run, st = _run_sweep(B, spec, {1, 7}, True, also_bf16_out=True, min_attention_checked=1)
+    print(f"pages of {page_tokens} tokens (llama shape, 4k): planted recall {_recall(spec, st):.2f}, {stats}")
+
+
+@pytest.mark.parametrize("page_tokens", [64, 128])
+def test_larger_cache_pages_off_the_page_boundary(B, page_tokens):
+    """A step that starts in the middle of a 64- or 128-token page (after a ragged step of 37
+    tokens): the pair kernel loads the partly filled last page whole and masks its tail; compared
+    with the oracle and with the general kernel."""
+    import torch
+    spec = wl.llama3_8b_layer().replace(context=4096, n_planted=0, page_tokens=page_tokens)
+    cfg = B.make_config(spec, out_dtype=B.F32)
+    st = B.RetrievalState(cfg, page_table=wl.shuffled_page_table(spec, spec.context)[None, :])
+    run = pu.OracleRunner(spec)
+    out = torch.zeros(spec.window, spec.n_q_heads, spec.head_dim, device="cuda")
+    for t, nt in [(0, 512), (1, 512), (2, 37), (3, 128), (4, 256)]:
+        q = wl.gen_q(spec, 0, t)[:nt]
+        k, v = wl.gen_kv(spec, 0, t)
+        k, v = k[:nt], v[:nt]
+        res = run.step(q, k, v, attention=t >= 3)
+        o = out[:nt]
+        dq, dk, dv = pu.to_device(q[None], spec), pu.to_device(k[None], spec), pu.to_device(v[None], spec)
+        p0 = st.host_pos0[0]
+        st.step(dq, dk, dv, o, n_tokens=nt, advance=False)
+        torch.cuda.synchronize()
+        assert int(st.status.item()) == 0
+        if t >= 3:
+            assert p0 % page_tokens != 0
+            assert pu.compare_selection(pu.to_numpy(st.sel_idx[0]).astype(np.int64), int(st.sel_count.item()), res,
+                                        f"step {t}") == 0
+            pu.assert_attention(pu.to_numpy(o), res["out"], f"p0 = {p0}, pages of {page_tokens}, pair kernel")
+            c2 = B.make_config(spec, out_dtype=B.F32, attention_kernel=B.ATTN_GENERAL)
+            o2 = torch.full_like(o, float("nan"))
+            B.retrieval_attention(c2, st.batch, dq, dk, dv, nt, st.k_pages, st.v_pages, st.page_table, st.pos0,
+                                  st.sel_idx, st.sel_count, o2, None, st.status)
+            torch.cuda.synchronize()
+            pu.assert_attention(pu.to_numpy(o2), res["out"], f"p0 = {p0}, pages of {page_tokens}, general kernel")
+        st.set_positions([p0 + nt])
+    assert int(st.status.item()) == 0
