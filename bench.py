@@ -551,7 +551,8 @@ def run_ours(args):
                         "select_cutoff": pick(s32, "select_cutoff"), "append": pick(s32, "append")},
             "decode16": {"workload": d16["workload"], "score_select": pick(d16, "score_select"),
                          "score_blocks": pick(d16, "score_blocks"), "select_cutoff": pick(d16, "select_cutoff"),
-                         "attention_decode": pick(d16, "attention_decode"), "keys_per_head": d16["keys_per_head"]},
+                         "attention_decode": pick(d16, "attention_decode"), "keys_per_head": d16["keys_per_head"],
+                         "model_step_32_layers": d16["stages"]["model_step_32_layers"]},
             "score_full_decode_step": sfull, "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
             "cold_l2": "512 MB read through L2 before every timed launch; median of 20 launches"}
         secondary["long131k"] = measure_long131k(device, peaks)
@@ -878,6 +879,54 @@ def measure_decode16(iters, dev, decode_splits=1):
         us, us_min = _time_stage(fn, iters, flush)
         res[name] = {"us": us, "min_us": us_min, "bytes": nbytes, "GBps": nbytes / us / 1e3,
                      "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+    # ---- a whole decode step of a 32-layer model with the paper's decode probe q^t (Sec. 4.2): per
+    # layer probe -> score -> cut-off / select -> decode attention -> append of the token, the layers
+    # rotating over the physical pools; enqueued call by call, and captured once into a CUDA graph.
+    n_model_layers = 32
+
+    def layer_step(l):
+        st = states[l % n_pools]
+        B.probe_query(cfg, st.batch, q, 1, None, st.probe_qh, st.probe_kv, st.status)
+        B.score_select(cfg, st.batch, st.probe_kv, st.repr_k, st.repr_inv_norm, st.n_cand, st.budget_state, st.scores,
+                       st.theta, st.sel_idx, st.sel_count, st.budget_real, st.status)
+        if ws is None:
+            B.retrieval_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                                  st.sel_count, out, None, st.status)
+        else:
+            B.decode_attention(cfg, st.batch, q, k, v, 1, st.k_pages, st.v_pages, st.page_table, st.pos0, st.sel_idx,
+                               st.sel_count, out, None, decode_splits, ws, st.status)
+        B.append_window(cfg, st.batch, k, v, 1, st.pos0, st.k_pages, st.v_pages, st.page_table, st.repr_k,
+                        st.repr_inv_norm, st.status)
+
+    def model_step():
+        for l in range(n_model_layers):
+            layer_step(l)
+
+    def time_model_step(fn):
+        for _ in range(2):
+            fn()
+        ts = []
+        for _ in range(max(5, iters // 2)):
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * a.elapsed_time(b))
+        return float(np.median(ts)), float(np.min(ts))
+
+    eager_us, eager_min = time_model_step(model_step)
+    step_graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(step_graph):
+        model_step()
+    graph_us, graph_min = time_model_step(step_graph.replay)
+    step_bytes = n_model_layers * (score_bytes + att_bytes)
+    res["model_step_32_layers"] = {
+        "us_graph": graph_us, "min_us_graph": graph_min, "us_eager": eager_us, "min_us_eager": eager_min,
+        "us_per_layer_graph": graph_us / n_model_layers, "tokens_per_s": S / (graph_us * 1e-6),
+        "bytes": step_bytes, "GBps": step_bytes / graph_us / 1e3,
+        "frac_of_measured_hbm": step_bytes / graph_us / 1e3 / peaks["hbm_gbs"],
+        "note": "probe q^t -> score -> cut-off / select -> decode attention -> append per layer, 32 layers over "
+                f"{n_pools} physical pools (their tables and pages are larger than L2), no flush between layers"}
     assert all(int(st.status.item()) == 0 for st in states)
     return {"workload": f"decode16: 16 sequences, contexts {int(ctx.min())}..{int(ctx.max())}, 1 token per step, "
                         f"one layer per launch, {n_pools} layer pools rotated",
